@@ -1,0 +1,229 @@
+/*
+ * nb.h - C ABI of the Non-blocking SGD aggregate-and-update library (CUDA, sm_100a).
+ *
+ * The library runs, on ONE GPU, the per-iteration aggregate-and-update of Non-blocking SGD
+ * (He & Dube, "Accelerating Parallel Stochastic Gradient Descent via Non-blocking Mini-batches")
+ * for K learners that are held as a batch dimension in device memory:
+ *
+ *   1. every learner i sums the gradients of the n_i mini-batches it finished before the fastest
+ *      learner raised the terminal signal; the unfinished ones are abandoned   (Alg. 1 inner loop;
+ *      Sec. 3.2 "Compute gradients"; Eq. 19);
+ *   2. the sum is scaled by a per-learner factor s_i                            (Sec. 3.2 "Adjust
+ *      learning rate"; Alg. 2 update step);
+ *   3. the learners' models are combined through a mixing matrix W:
+ *      x_half_i = sum_j W_ij x_j                                                (Alg. 2 averaging step;
+ *      Eq. 4-5 for the all-reduce mean; Eq. 6 for D-PSGD; Sec. 6.1 for MATCHA's activated matchings);
+ *   4. a momentum-SGD step follows: v_i <- mom v_i + s_i acc_i, x_i <- x_half_i - lr v_i
+ *      (Alg. 2 update step; momentum is this library's addition, mom = 0 gives the paper's rule).
+ *
+ * Notation: the paper writes P for the number of learners, d for the parameter dimension and N for
+ * the number of mini-batches; this header uses K learners, P parameters, M mini-batches.
+ *
+ * Conventions for every entry point
+ *   - returns an nb_status; nothing throws, aborts or prints across the boundary;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream); device work
+ *     is enqueued on it and the call returns without waiting, except where stated;
+ *   - pointers marked "host" are read or written on the CPU before the call returns and are never
+ *     retained; pointers marked "device" must stay valid until `stream` has passed the call's work;
+ *   - a context is bound to the device that was current at nb_create and must be used from one host
+ *     thread at a time;
+ *   - a CUDA failure is reported as NB_ERR_CUDA and is sticky for that context.
+ */
+#ifndef NB_H_
+#define NB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NB_MAX_K 64          /* learners                                                     */
+#define NB_MAX_MATCHINGS 32  /* matchings of a MATCHA topology (activation bits fit a word)  */
+#define NB_MAX_NNZ 1024      /* non-zeros of a sparse mixing matrix                          */
+
+typedef struct nb_ctx nb_ctx; /* opaque; owned by the library */
+
+enum nb_status {
+  NB_OK = 0,
+  NB_ERR_ARG = -1,         /* invalid argument (nb_last_error says which)               */
+  NB_ERR_STATE = -2,       /* call order violated (e.g. nb_step without nb_accumulate)  */
+  NB_ERR_CUDA = -3,        /* a CUDA call failed; sticky                                 */
+  NB_ERR_NOMEM = -4,       /* device or host allocation failed                           */
+  NB_ERR_UNSUPPORTED = -5  /* valid request outside the library's limits                 */
+};
+
+/* How the learners are combined (step 3 above). */
+enum nb_variant {
+  NB_ALLREDUCE = 0,   /* W = (1/K) 1 1^T: mean over learners (Eq. 4-5)                              */
+  NB_DPSGD = 1,       /* fixed sparse doubly-stochastic W (Eq. 6; Alg. 2)                           */
+  NB_MATCHA = 2,      /* W(t) = I - alpha * sum of the Laplacians of the matchings active at t      */
+  NB_CENTRALIZED = 3  /* one parameter-server model shared by all learners (Alg. 3)                 */
+};
+
+enum nb_dtype { NB_F32 = 0, NB_BF16 = 1 }; /* element type of the gradient stream */
+
+enum nb_topology_kind {
+  NB_TOPO_FULL = 0,           /* complete graph, W_ij = 1/K                                          */
+  NB_TOPO_RING = 1,           /* W_ii = W_i,i+1 = W_i,i-1 = 1/3 (indices mod K)                      */
+  NB_TOPO_CSR = 2,            /* explicit W in CSR form                                              */
+  NB_TOPO_MATCHINGS = 3,      /* explicit matchings (partner table)                                  */
+  NB_TOPO_RANDOM_REGULAR = 4  /* seeded random `degree`-regular graph, greedily split into matchings */
+};
+
+/* Topology description, host memory, copied by the callee.  Unused fields are ignored. */
+typedef struct nb_topology {
+  int32_t kind;            /* nb_topology_kind                                                     */
+  int32_t degree;          /* RANDOM_REGULAR: vertex degree (K*degree even, degree < K)            */
+  uint64_t seed;           /* RANDOM_REGULAR: graph seed; MATCHA: also seeds the activation draws  */
+  const int32_t *row_ptr;  /* CSR: [K+1]                                                           */
+  const int32_t *col_idx;  /* CSR: [row_ptr[K]], any order inside a row                            */
+  const float *val;        /* CSR: [row_ptr[K]]; rows and columns must sum to 1 within 1e-5        */
+  int32_t n_matchings;     /* MATCHINGS: number of matchings, <= NB_MAX_MATCHINGS                  */
+  const int32_t *partner;  /* MATCHINGS: [n_matchings*K], partner[c*K+v] = v's partner, -1 = none  */
+  float alpha;             /* MATCHA: W = I - alpha * sum_active L_j                               */
+  float act_prob;          /* MATCHA: each matching is active with this probability, per step      */
+} nb_topology;
+
+/* nb_set_option keys and values */
+enum nb_option {
+  NB_OPT_NORM = 0,  /* NB_NORM_MEAN (default) | NB_NORM_PAPER */
+  NB_OPT_ORDER = 1  /* NB_ORDER_MIX_THEN_UPDATE (default) | NB_ORDER_UPDATE_THEN_MIX */
+};
+enum nb_norm {
+  NB_NORM_MEAN = 0,  /* s_i = 1/n_i: mean of the finished mini-batch gradients (s_i = 0 if n_i = 0)        */
+  NB_NORM_PAPER = 1  /* s_i = n_i/M: the learning-rate adjustment eta*n/N of Alg. 2 applied to the sum     */
+};
+enum nb_order {
+  NB_ORDER_MIX_THEN_UPDATE = 0, /* Alg. 2: x_i <- sum_j W_ij x_j - lr v_i                                   */
+  NB_ORDER_UPDATE_THEN_MIX = 1  /* Eq. 4-6: x_i <- sum_j W_ij (x_j - lr v_j)                                */
+};
+
+/* ------------------------------------------------------------------------------------------------
+ * Host straggler simulator: stands in for the terminal signal of Alg. 1 (the first learner to
+ * finish its M mini-batches ends the iteration; the others abandon what they have not finished).
+ * One mini-batch time tau_i per learner per iteration (Sec. 4.1), constant speed inside an
+ * iteration (Sec. 4.3): n_i = max(1, #{j in 1..M : j*tau_i <= M*min_i tau_i}).
+ * Pure functions of (configuration, step): no context, no GPU.
+ * ---------------------------------------------------------------------------------------------- */
+enum nb_straggler_model {
+  NB_STRAG_UNIFORM_COUNT = 0,       /* n_i uniform on {1..M}; no parameters                               */
+  NB_STRAG_SHIFTED_EXP = 1,         /* tau_i = 1 + Exp(mean params[0])                                    */
+  NB_STRAG_SHIFTED_EXP_SLOWSET = 2  /* floor(params[0]*K) learners, re-drawn every step, have mean        */
+                                    /* params[1]; the rest have mean params[2]                             */
+};
+typedef struct nb_straggler {
+  int32_t model;     /* nb_straggler_model */
+  uint64_t seed;
+  double params[4];
+} nb_straggler;
+
+/* finished: host out [K].  mask: host out [K*M] (mask[i*M+m] = m < n_i) or NULL.
+ * tau: host out [K] mini-batch times, or NULL (written as 0 for UNIFORM_COUNT).
+ * Errors: NB_ERR_ARG for K<1, K>NB_MAX_K, M<1, unknown model, negative means. */
+int nb_straggler_sample(const nb_straggler *cfg, int K, int M, int64_t step, int32_t *finished,
+                        uint8_t *mask, double *tau);
+
+/* ------------------------------------------------------------------------------------------------
+ * Host topology helpers (no context, no GPU).
+ * ---------------------------------------------------------------------------------------------- */
+
+/* Matchings of a MATCHINGS or RANDOM_REGULAR topology.  partner: host out [NB_MAX_MATCHINGS*K]
+ * (first n*K entries written); n_matchings: host out; attempts: host out or NULL (graph draws
+ * rejected + 1).  Errors: NB_ERR_ARG for an impossible degree, a partner table that is not an
+ * involution or repeats an edge; NB_ERR_UNSUPPORTED if more than NB_MAX_MATCHINGS are needed. */
+int nb_topology_matchings(const nb_topology *topo, int K, int32_t *partner, int32_t *n_matchings,
+                          int32_t *attempts);
+
+/* The mixing matrix a context created with (variant, topo, K) uses at `step`, dense row-major
+ * host out [K*K]; bits: host out or NULL, the MATCHA activation word (bit j = matching j active).
+ * Same validation as nb_create. */
+int nb_mixing_matrix(const nb_topology *topo, int variant, int K, int64_t step, float *W_dense,
+                     uint32_t *bits);
+
+/* ------------------------------------------------------------------------------------------------
+ * Context
+ * ---------------------------------------------------------------------------------------------- */
+
+/* Creates a context on the current device: K learners, P parameters each, M mini-batches per
+ * batch; allocates the models X[K,P], the momentum V[K,P] (zeroed) and the accumulator acc[K,P]
+ * in fp32 (NB_CENTRALIZED: one model and one momentum vector; acc still [K,P]).
+ * topo may be NULL for NB_ALLREDUCE and NB_CENTRALIZED.  NB_DPSGD takes RING, FULL or CSR;
+ * NB_MATCHA takes MATCHINGS or RANDOM_REGULAR.
+ * Errors: NB_ERR_ARG (K<1, P<1, M<1, bad topology, W not doubly stochastic within 1e-5),
+ * NB_ERR_UNSUPPORTED (K>NB_MAX_K, nnz>NB_MAX_NNZ), NB_ERR_NOMEM, NB_ERR_CUDA.  *out is NULL on error. */
+int nb_create(nb_ctx **out, int K, int64_t P, int M, float lr, float mom, int variant,
+              const nb_topology *topo);
+
+/* Frees everything the context owns (waits for the device first).  NULL is accepted. */
+int nb_destroy(nb_ctx *c);
+
+/* Last error text of this context (or of the last failed nb_create when c is NULL). */
+const char *nb_last_error(const nb_ctx *c);
+
+int nb_set_option(nb_ctx *c, int key, int64_t value);
+int nb_set_lr(nb_ctx *c, float lr);
+
+/* Loads the models: per_learner = 0: x0[P] is given to every learner ("initialize local models
+ * with the same initialization", Alg. 1); per_learner = 1: x0[K,P] dense.  x0: host or device.
+ * Zeroes the momentum and the step counter.  NB_CENTRALIZED accepts only per_learner = 0. */
+int nb_set_params(nb_ctx *c, const float *x0, int per_learner, void *stream);
+
+/* Masked accumulate (step 1): acc[i,p] = sum_{m < finished[i]} grads[i,m,p], fp32 accumulation in
+ * ascending m; rows m >= finished[i] are never read.
+ * grads: device, element (i,m,p) at grads[i*ld_k + m*ld_m + p], dtype NB_F32 or NB_BF16;
+ * ld_m, ld_k in elements, 0 = dense (ld_m = P, ld_k = M*P).  The 128-bit path needs grads, ld_m
+ * and ld_k aligned to 4 elements; anything else runs a scalar kernel on the GPU.
+ * finished: host [K], each in [0, M].  Errors: NB_ERR_ARG. */
+int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
+                  const int32_t *finished, void *stream);
+
+/* Steps 2-4 on what the last nb_accumulate stored; advances the step counter.
+ * NB_ERR_STATE if there has been no nb_accumulate since the last step. */
+int nb_step(nb_ctx *c, void *stream);
+
+/* Steps 1-4 in a single pass over the gradient stream without the acc round trip.  The result is
+ * bit-identical to nb_accumulate followed by nb_step.  Arguments as nb_accumulate. */
+int nb_step_fused(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
+                  const int32_t *finished, void *stream);
+
+/* As nb_step_fused with the gradient stream in HOST memory (pinned for speed): copies only the
+ * finished mini-batch rows into a staging buffer the context allocates on first use ([K,M,P]
+ * elements of the widest dtype seen), runs the fused step and, when mean_out is not NULL, writes
+ * the mean model (Alg. 1 "Output") to host memory mean_out[P].  Waits for `stream` before it
+ * returns. */
+int nb_step_fused_host(nb_ctx *c, const void *grads_host, int dtype, int64_t ld_m, int64_t ld_k,
+                       const int32_t *finished, float *mean_out, void *stream);
+
+/* Outputs.  dst is host or device memory, dense.  Copies to pageable host memory wait for `stream`. */
+int nb_get_params(nb_ctx *c, float *dst /* [K,P] ([P] for NB_CENTRALIZED) */, void *stream);
+int nb_get_momentum(nb_ctx *c, float *dst /* as nb_get_params */, void *stream);
+int nb_get_accumulator(nb_ctx *c, float *dst /* [K,P] */, void *stream);
+/* Average of all learners' models (Alg. 1 / Alg. 2 "Output"), summed in ascending learner order. */
+int nb_get_mean_params(nb_ctx *c, float *dst /* [P] */, void *stream);
+
+/* Checkpoint / resume: loads models, momentum (dense, host or device, shaped as nb_get_params
+ * returns them) and the step counter.  All randomness is a function of (seed, step), so a restored
+ * run continues bit-identically. */
+int nb_set_state(nb_ctx *c, int64_t step, const float *X, const float *V, void *stream);
+int nb_get_step(const nb_ctx *c, int64_t *step);
+
+/* The mixing matrix this context uses at `step` (host-side computation), dense host out [K*K]. */
+int nb_get_W(nb_ctx *c, int64_t step, float *W_dense);
+/* MATCHA: the activation word the host computes for `step`. */
+int nb_get_matcha_activation(nb_ctx *c, int64_t step, uint32_t *bits);
+/* MATCHA: what the DEVICE-side builder produced for the most recent step: its activation word and
+ * its W, densified (host out [K*K]).  Waits for `stream`.  NB_ERR_STATE before the first step. */
+int nb_get_device_mixing(nb_ctx *c, uint32_t *bits, float *W_dense, void *stream);
+
+/* Counters of the most recent step: sum of finished counts, algorithmic bytes
+ * P*(e_g*sum n_i + 16*K) (e_g = bytes per gradient element; NB_CENTRALIZED: 16 instead of 16*K),
+ * and the number of kernels this library has launched on this context so far. */
+int nb_get_stats(const nb_ctx *c, int64_t *sum_finished, double *algorithmic_bytes,
+                 int64_t *kernel_launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NB_H_ */

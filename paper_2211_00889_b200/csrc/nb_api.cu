@@ -1,0 +1,508 @@
+// C ABI of the library: context management, argument validation, launches.  See include/nb.h for
+// the contract of every entry point.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "nb_internal.h"
+#include "nb_kernels.h"
+
+struct nb_ctx {
+  int device = 0;
+  int K = 0, M = 0, rows = 0;  // rows = model rows held (K, or 1 for NB_CENTRALIZED)
+  int64_t P = 0, ldx = 0;
+  float lr = 0.f, mom = 0.f;
+  int variant = NB_ALLREDUCE, norm = NB_NORM_MEAN, order = NB_ORDER_MIX_THEN_UPDATE;
+  nb::Mixing mx;
+  float *X = nullptr, *V = nullptr, *acc = nullptr, *d_mean = nullptr;
+  nb::MixTable *d_mix = nullptr;
+  int32_t *d_partner = nullptr;
+  void *staging = nullptr;
+  size_t staging_bytes = 0;
+  int64_t step = 0;
+  bool acc_fresh = false, device_mix_valid = false;
+  int32_t n_acc[NB_MAX_K] = {0};
+  int acc_esize = 4;
+  int64_t sum_finished = 0, launches = 0;
+  double alg_bytes = 0.0;
+  int sticky = NB_OK;
+  std::string err;
+};
+
+namespace {
+
+thread_local std::string g_create_err;
+
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+
+int fail(nb_ctx *c, int code, const std::string &msg) {
+  if (c) {
+    c->err = msg;
+    if (code == NB_ERR_CUDA) c->sticky = NB_ERR_CUDA;
+  } else {
+    g_create_err = msg;
+  }
+  return code;
+}
+
+int cuda_fail(nb_ctx *c, cudaError_t e, const char *what) {
+  return fail(c, e == cudaErrorMemoryAllocation ? NB_ERR_NOMEM : NB_ERR_CUDA,
+              std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+#define NB_CUDA(c, call)                                       \
+  do {                                                         \
+    cudaError_t e__ = (call);                                  \
+    if (e__ != cudaSuccess) return cuda_fail((c), e__, #call); \
+  } while (0)
+
+#define NB_ENTER(c)                                                       \
+  if (!(c)) return NB_ERR_ARG;                                            \
+  if ((c)->sticky != NB_OK) return (c)->sticky;                           \
+  DeviceGuard guard__((c)->device)
+
+bool is_device_pointer(const void *p) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged;
+}
+
+// Validates the gradient-stream description and the finished counts; fills the step arguments.
+int fill_step_args(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k, const int32_t *finished,
+                   nb::StepArgs *a, int *esize) {
+  if (!grads) return fail(c, NB_ERR_ARG, "grads is NULL");
+  if (!finished) return fail(c, NB_ERR_ARG, "finished is NULL");
+  if (dtype != NB_F32 && dtype != NB_BF16) return fail(c, NB_ERR_ARG, "dtype must be NB_F32 or NB_BF16");
+  const int es = dtype == NB_F32 ? 4 : 2;
+  if (ld_m == 0) ld_m = c->P;
+  if (ld_k == 0) ld_k = (int64_t)c->M * ld_m;
+  if (ld_m < c->P) return fail(c, NB_ERR_ARG, "ld_m is smaller than P");
+  if (ld_k < (int64_t)(c->M - 1) * ld_m + c->P) return fail(c, NB_ERR_ARG, "ld_k is too small for M rows of pitch ld_m");
+  int64_t sum = 0;
+  for (int i = 0; i < c->K; ++i) {
+    if (finished[i] < 0 || finished[i] > c->M)
+      return fail(c, NB_ERR_ARG, "finished[" + std::to_string(i) + "] is outside [0, M]");
+    sum += finished[i];
+  }
+  std::memset(a, 0, sizeof(*a));
+  a->X = c->X;
+  a->V = c->V;
+  a->acc = c->acc;
+  a->G = grads;
+  a->mix = c->d_mix;
+  a->ldx = c->ldx;
+  a->ld_m = ld_m;
+  a->ld_k = ld_k;
+  a->P = c->P;
+  a->K = c->K;
+  a->M = c->M;
+  a->g_aligned = ((uintptr_t)grads % (size_t)(4 * es) == 0) && (ld_m % 4 == 0) && (ld_k % 4 == 0);
+  for (int i = 0; i < c->K; ++i) a->n[i] = finished[i];
+  *esize = es;
+  (void)sum;
+  return NB_OK;
+}
+
+// Scalars, scale factors and mixing mode: the part of the arguments the step (not the accumulate) needs.
+void fill_update_args(nb_ctx *c, nb::StepArgs *a) {
+  a->lr = c->lr;
+  a->mom = c->mom;
+  a->inv_K = 1.0f / (float)c->K;
+  a->order = c->order;
+  a->mean_mode = (c->variant == NB_ALLREDUCE) ? 1 : 0;
+  a->mix_slots = 0;
+  if (c->variant == NB_DPSGD) a->mix_slots = (int32_t)c->mx.col.size();
+  if (c->variant == NB_MATCHA) a->mix_slots = c->K * (1 + c->mx.n_matchings);
+  for (int i = 0; i < c->K; ++i) {
+    const int n = a->n[i];
+    if (c->norm == NB_NORM_MEAN) a->s[i] = n > 0 ? 1.0f / (float)n : 0.0f;
+    else a->s[i] = (float)n / (float)c->M;
+  }
+}
+
+void record_stats(nb_ctx *c, const nb::StepArgs &a, int esize) {
+  int64_t sum = 0;
+  for (int i = 0; i < c->K; ++i) sum += a.n[i];
+  c->sum_finished = sum;
+  c->alg_bytes = (double)c->P * ((double)esize * (double)sum + 16.0 * (double)c->rows);
+}
+
+// MATCHA: rebuild W on the device for the current step (K3), ahead of the step kernel in `st`.
+int build_device_mixing(nb_ctx *c, cudaStream_t st) {
+  if (c->variant != NB_MATCHA) return NB_OK;
+  nb::MatchaArgs m;
+  m.mix = c->d_mix;
+  m.partner = c->d_partner;
+  m.seed = c->mx.seed;
+  m.thr = nb::activation_threshold(c->mx.act_prob);
+  m.step = c->step;
+  m.K = c->K;
+  m.n_matchings = c->mx.n_matchings;
+  m.alpha = c->mx.alpha;
+  NB_CUDA(c, nb::launch_matcha_build(m, st));
+  c->launches++;
+  c->device_mix_valid = true;
+  return NB_OK;
+}
+
+int run_update(nb_ctx *c, nb::StepArgs *a, int src, cudaStream_t st) {
+  fill_update_args(c, a);
+  if (c->variant == NB_CENTRALIZED) {
+    NB_CUDA(c, nb::launch_centralized(*a, src, st));
+  } else {
+    int rc = build_device_mixing(c, st);
+    if (rc != NB_OK) return rc;
+    NB_CUDA(c, nb::launch_step(*a, src, st));
+  }
+  c->launches++;
+  c->step++;
+  c->acc_fresh = false;
+  return NB_OK;
+}
+
+// dense [rows, P] <-> pitched [rows, ldx]
+int copy_rows_out(nb_ctx *c, float *dst, const float *src, int rows, cudaStream_t st) {
+  if (!dst) return fail(c, NB_ERR_ARG, "dst is NULL");
+  for (int r = 0; r < rows; ++r)
+    NB_CUDA(c, cudaMemcpyAsync(dst + (int64_t)r * c->P, src + (int64_t)r * c->ldx, sizeof(float) * (size_t)c->P,
+                               cudaMemcpyDefault, st));
+  if (!is_device_pointer(dst)) NB_CUDA(c, cudaStreamSynchronize(st));
+  return NB_OK;
+}
+int copy_rows_in(nb_ctx *c, float *dst, const float *src, int rows, cudaStream_t st) {
+  for (int r = 0; r < rows; ++r)
+    NB_CUDA(c, cudaMemcpyAsync(dst + (int64_t)r * c->ldx, src + (int64_t)r * c->P, sizeof(float) * (size_t)c->P,
+                               cudaMemcpyDefault, st));
+  if (!is_device_pointer(src)) NB_CUDA(c, cudaStreamSynchronize(st));
+  return NB_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *nb_last_error(const nb_ctx *c) { return c ? c->err.c_str() : g_create_err.c_str(); }
+
+int nb_create(nb_ctx **out, int K, int64_t P, int M, float lr, float mom, int variant, const nb_topology *topo) {
+  if (!out) return NB_ERR_ARG;
+  *out = nullptr;
+  if (K < 1) return fail(nullptr, NB_ERR_ARG, "K must be >= 1");
+  if (P < 1) return fail(nullptr, NB_ERR_ARG, "P must be >= 1");
+  if (M < 1) return fail(nullptr, NB_ERR_ARG, "M must be >= 1");
+  if (variant < NB_ALLREDUCE || variant > NB_CENTRALIZED) return fail(nullptr, NB_ERR_ARG, "unknown variant");
+  nb::Mixing mx;
+  std::string err;
+  int rc = nb::build_mixing(topo, variant, K, &mx, &err);
+  if (rc != NB_OK) return fail(nullptr, rc, err);
+
+  nb_ctx *c = new (std::nothrow) nb_ctx;
+  if (!c) return fail(nullptr, NB_ERR_NOMEM, "host allocation failed");
+  c->K = K;
+  c->P = P;
+  c->M = M;
+  c->lr = lr;
+  c->mom = mom;
+  c->variant = variant;
+  c->rows = variant == NB_CENTRALIZED ? 1 : K;
+  c->ldx = (P + 31) / 32 * 32;  // rows start on 128-byte boundaries
+  c->mx = mx;
+
+  auto bail = [&](cudaError_t e, const char *what) {
+    int code = cuda_fail(nullptr, e, what);
+    cudaGetLastError();
+    nb_destroy(c);
+    return code;
+  };
+  cudaError_t e;
+  if ((e = cudaGetDevice(&c->device)) != cudaSuccess) return bail(e, "cudaGetDevice");
+  if ((e = nb::configure_kernels()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute");
+  const size_t model_bytes = sizeof(float) * (size_t)c->rows * (size_t)c->ldx;
+  const size_t acc_bytes = sizeof(float) * (size_t)K * (size_t)c->ldx;
+  if ((e = cudaMalloc(&c->X, model_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(X)");
+  if ((e = cudaMalloc(&c->V, model_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(V)");
+  if ((e = cudaMalloc(&c->acc, acc_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(acc)");
+  if ((e = cudaMemset(c->X, 0, model_bytes)) != cudaSuccess) return bail(e, "cudaMemset(X)");
+  if ((e = cudaMemset(c->V, 0, model_bytes)) != cudaSuccess) return bail(e, "cudaMemset(V)");
+  if ((e = cudaMemset(c->acc, 0, acc_bytes)) != cudaSuccess) return bail(e, "cudaMemset(acc)");
+  if (variant == NB_DPSGD || variant == NB_MATCHA) {
+    if ((e = cudaMalloc(&c->d_mix, sizeof(nb::MixTable))) != cudaSuccess) return bail(e, "cudaMalloc(mix)");
+    nb::MixTable *h = new (std::nothrow) nb::MixTable;
+    if (!h) { nb_destroy(c); return fail(nullptr, NB_ERR_NOMEM, "host allocation failed"); }
+    std::memset(h, 0, sizeof(*h));
+    if (variant == NB_DPSGD) {
+      for (int i = 0; i < K; ++i) { h->row_beg[i] = mx.row_ptr[i]; h->row_end[i] = mx.row_ptr[i + 1]; }
+      for (size_t q = 0; q < mx.col.size(); ++q) { h->col[q] = mx.col[q]; h->val[q] = mx.val[q]; }
+      h->n_slots = (int32_t)mx.col.size();
+    }
+    e = cudaMemcpy(c->d_mix, h, sizeof(*h), cudaMemcpyHostToDevice);
+    delete h;
+    if (e != cudaSuccess) return bail(e, "cudaMemcpy(mix)");
+  }
+  if (variant == NB_MATCHA && mx.n_matchings > 0) {
+    const size_t pb = sizeof(int32_t) * mx.partner.size();
+    if ((e = cudaMalloc(&c->d_partner, pb)) != cudaSuccess) return bail(e, "cudaMalloc(partner)");
+    if ((e = cudaMemcpy(c->d_partner, mx.partner.data(), pb, cudaMemcpyHostToDevice)) != cudaSuccess)
+      return bail(e, "cudaMemcpy(partner)");
+  }
+  *out = c;
+  return NB_OK;
+}
+
+int nb_destroy(nb_ctx *c) {
+  if (!c) return NB_OK;
+  DeviceGuard guard(c->device);
+  cudaDeviceSynchronize();
+  cudaFree(c->X);
+  cudaFree(c->V);
+  cudaFree(c->acc);
+  cudaFree(c->d_mean);
+  cudaFree(c->d_mix);
+  cudaFree(c->d_partner);
+  cudaFree(c->staging);
+  cudaGetLastError();
+  delete c;
+  return NB_OK;
+}
+
+int nb_set_option(nb_ctx *c, int key, int64_t value) {
+  NB_ENTER(c);
+  if (key == NB_OPT_NORM) {
+    if (value != NB_NORM_MEAN && value != NB_NORM_PAPER) return fail(c, NB_ERR_ARG, "unknown norm");
+    c->norm = (int)value;
+    return NB_OK;
+  }
+  if (key == NB_OPT_ORDER) {
+    if (value != NB_ORDER_MIX_THEN_UPDATE && value != NB_ORDER_UPDATE_THEN_MIX) return fail(c, NB_ERR_ARG, "unknown order");
+    c->order = (int)value;
+    return NB_OK;
+  }
+  return fail(c, NB_ERR_ARG, "unknown option key");
+}
+
+int nb_set_lr(nb_ctx *c, float lr) {
+  NB_ENTER(c);
+  c->lr = lr;
+  return NB_OK;
+}
+
+int nb_set_params(nb_ctx *c, const float *x0, int per_learner, void *stream) {
+  NB_ENTER(c);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!x0) return fail(c, NB_ERR_ARG, "x0 is NULL");
+  if (per_learner != 0 && per_learner != 1) return fail(c, NB_ERR_ARG, "per_learner must be 0 or 1");
+  if (per_learner && c->variant == NB_CENTRALIZED) return fail(c, NB_ERR_ARG, "NB_CENTRALIZED holds one model");
+  if (per_learner) {
+    int rc = copy_rows_in(c, c->X, x0, c->rows, st);
+    if (rc != NB_OK) return rc;
+  } else {
+    int rc = copy_rows_in(c, c->X, x0, 1, st);
+    if (rc != NB_OK) return rc;
+    for (int r = 1; r < c->rows; ++r)
+      NB_CUDA(c, cudaMemcpyAsync(c->X + (int64_t)r * c->ldx, c->X, sizeof(float) * (size_t)c->P, cudaMemcpyDeviceToDevice, st));
+  }
+  NB_CUDA(c, cudaMemsetAsync(c->V, 0, sizeof(float) * (size_t)c->rows * (size_t)c->ldx, st));
+  c->step = 0;
+  c->acc_fresh = false;
+  return NB_OK;
+}
+
+int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k, const int32_t *finished,
+                  void *stream) {
+  NB_ENTER(c);
+  nb::StepArgs a;
+  int es = 4;
+  int rc = fill_step_args(c, grads, dtype, ld_m, ld_k, finished, &a, &es);
+  if (rc != NB_OK) return rc;
+  NB_CUDA(c, nb::launch_accumulate(a, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16, (cudaStream_t)stream));
+  c->launches++;
+  std::memcpy(c->n_acc, a.n, sizeof(c->n_acc));
+  c->acc_esize = es;
+  c->acc_fresh = true;
+  return NB_OK;
+}
+
+int nb_step(nb_ctx *c, void *stream) {
+  NB_ENTER(c);
+  if (!c->acc_fresh) return fail(c, NB_ERR_STATE, "nb_step needs an nb_accumulate since the last step");
+  nb::StepArgs a;
+  std::memset(&a, 0, sizeof(a));
+  a.X = c->X;
+  a.V = c->V;
+  a.acc = c->acc;
+  a.mix = c->d_mix;
+  a.ldx = c->ldx;
+  a.P = c->P;
+  a.K = c->K;
+  a.M = c->M;
+  a.g_aligned = 1;
+  std::memcpy(a.n, c->n_acc, sizeof(a.n));
+  record_stats(c, a, c->acc_esize);
+  return run_update(c, &a, nb::kSrcAcc, (cudaStream_t)stream);
+}
+
+int nb_step_fused(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k, const int32_t *finished,
+                  void *stream) {
+  NB_ENTER(c);
+  nb::StepArgs a;
+  int es = 4;
+  int rc = fill_step_args(c, grads, dtype, ld_m, ld_k, finished, &a, &es);
+  if (rc != NB_OK) return rc;
+  record_stats(c, a, es);
+  return run_update(c, &a, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16, (cudaStream_t)stream);
+}
+
+int nb_step_fused_host(nb_ctx *c, const void *grads_host, int dtype, int64_t ld_m, int64_t ld_k,
+                       const int32_t *finished, float *mean_out, void *stream) {
+  NB_ENTER(c);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!grads_host) return fail(c, NB_ERR_ARG, "grads_host is NULL");
+  if (!finished) return fail(c, NB_ERR_ARG, "finished is NULL");
+  if (dtype != NB_F32 && dtype != NB_BF16) return fail(c, NB_ERR_ARG, "dtype must be NB_F32 or NB_BF16");
+  const size_t es = dtype == NB_F32 ? 4 : 2;
+  if (ld_m == 0) ld_m = c->P;
+  if (ld_k == 0) ld_k = (int64_t)c->M * ld_m;
+  if (ld_m < c->P) return fail(c, NB_ERR_ARG, "ld_m is smaller than P");
+  for (int i = 0; i < c->K; ++i)
+    if (finished[i] < 0 || finished[i] > c->M) return fail(c, NB_ERR_ARG, "finished count outside [0, M]");
+  const int64_t ldg = (c->P + 31) / 32 * 32;  // staging pitch, elements
+  const size_t need = (size_t)c->K * (size_t)c->M * (size_t)ldg * es;
+  if (c->staging_bytes < need) {
+    NB_CUDA(c, cudaStreamSynchronize(st));
+    cudaFree(c->staging);
+    c->staging = nullptr;
+    c->staging_bytes = 0;
+    NB_CUDA(c, cudaMalloc(&c->staging, need));
+    c->staging_bytes = need;
+  }
+  // only the finished mini-batches cross the bus: the abandoned ones are never needed
+  for (int i = 0; i < c->K; ++i)
+    for (int m = 0; m < finished[i]; ++m) {
+      const char *src = (const char *)grads_host + ((size_t)i * (size_t)ld_k + (size_t)m * (size_t)ld_m) * es;
+      char *dst = (char *)c->staging + ((size_t)i * (size_t)c->M + (size_t)m) * (size_t)ldg * es;
+      NB_CUDA(c, cudaMemcpyAsync(dst, src, (size_t)c->P * es, cudaMemcpyHostToDevice, st));
+    }
+  int rc = nb_step_fused(c, c->staging, dtype, ldg, (int64_t)c->M * ldg, finished, stream);
+  if (rc != NB_OK) return rc;
+  if (mean_out) {
+    rc = nb_get_mean_params(c, mean_out, stream);
+    if (rc != NB_OK) return rc;
+  }
+  NB_CUDA(c, cudaStreamSynchronize(st));
+  return NB_OK;
+}
+
+int nb_get_params(nb_ctx *c, float *dst, void *stream) {
+  NB_ENTER(c);
+  return copy_rows_out(c, dst, c->X, c->rows, (cudaStream_t)stream);
+}
+
+int nb_get_momentum(nb_ctx *c, float *dst, void *stream) {
+  NB_ENTER(c);
+  return copy_rows_out(c, dst, c->V, c->rows, (cudaStream_t)stream);
+}
+
+int nb_get_accumulator(nb_ctx *c, float *dst, void *stream) {
+  NB_ENTER(c);
+  return copy_rows_out(c, dst, c->acc, c->K, (cudaStream_t)stream);
+}
+
+int nb_get_mean_params(nb_ctx *c, float *dst, void *stream) {
+  NB_ENTER(c);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!dst) return fail(c, NB_ERR_ARG, "dst is NULL");
+  const bool dev = is_device_pointer(dst);
+  float *out = dst;
+  if (!dev) {
+    if (!c->d_mean) NB_CUDA(c, cudaMalloc(&c->d_mean, sizeof(float) * (size_t)c->P));
+    out = c->d_mean;
+  }
+  NB_CUDA(c, nb::launch_mean(c->X, c->ldx, c->rows, c->P, out, st));
+  c->launches++;
+  if (!dev) {
+    NB_CUDA(c, cudaMemcpyAsync(dst, out, sizeof(float) * (size_t)c->P, cudaMemcpyDeviceToHost, st));
+    NB_CUDA(c, cudaStreamSynchronize(st));
+  }
+  return NB_OK;
+}
+
+int nb_set_state(nb_ctx *c, int64_t step, const float *X, const float *V, void *stream) {
+  NB_ENTER(c);
+  if (step < 0 || !X || !V) return fail(c, NB_ERR_ARG, "nb_set_state: step >= 0 and X, V required");
+  int rc = copy_rows_in(c, c->X, X, c->rows, (cudaStream_t)stream);
+  if (rc != NB_OK) return rc;
+  rc = copy_rows_in(c, c->V, V, c->rows, (cudaStream_t)stream);
+  if (rc != NB_OK) return rc;
+  c->step = step;
+  c->acc_fresh = false;
+  return NB_OK;
+}
+
+int nb_get_step(const nb_ctx *c, int64_t *step) {
+  if (!c || !step) return NB_ERR_ARG;
+  *step = c->step;
+  return NB_OK;
+}
+
+int nb_get_W(nb_ctx *c, int64_t step, float *W_dense) {
+  if (!c) return NB_ERR_ARG;
+  if (!W_dense || step < 0) return fail(c, NB_ERR_ARG, "nb_get_W: W_dense and step >= 0 required");
+  nb::dense_W(c->mx, step, W_dense, nullptr);
+  return NB_OK;
+}
+
+int nb_get_matcha_activation(nb_ctx *c, int64_t step, uint32_t *bits) {
+  if (!c) return NB_ERR_ARG;
+  if (!bits || step < 0) return fail(c, NB_ERR_ARG, "bits and step >= 0 required");
+  if (c->variant != NB_MATCHA) return fail(c, NB_ERR_STATE, "not a MATCHA context");
+  *bits = nb::matcha_bits(c->mx.seed, step, c->mx.n_matchings, nb::activation_threshold(c->mx.act_prob));
+  return NB_OK;
+}
+
+int nb_get_device_mixing(nb_ctx *c, uint32_t *bits, float *W_dense, void *stream) {
+  NB_ENTER(c);
+  if (c->variant != NB_MATCHA) return fail(c, NB_ERR_STATE, "not a MATCHA context");
+  if (!c->device_mix_valid) return fail(c, NB_ERR_STATE, "no step has run yet");
+  nb::MixTable *h = new (std::nothrow) nb::MixTable;
+  if (!h) return fail(c, NB_ERR_NOMEM, "host allocation failed");
+  cudaError_t e = cudaMemcpyAsync(h, c->d_mix, sizeof(*h), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) {
+    delete h;
+    return cuda_fail(c, e, "cudaMemcpyAsync(mix)");
+  }
+  if (bits) *bits = h->bits;
+  if (W_dense) {
+    const int K = c->K;
+    for (size_t q = 0; q < (size_t)K * K; ++q) W_dense[q] = 0.f;
+    for (int i = 0; i < K; ++i)
+      for (int e2 = h->row_beg[i]; e2 < h->row_end[i]; ++e2)
+        if (e2 >= 0 && e2 < NB_MAX_NNZ && h->col[e2] >= 0 && h->col[e2] < K) W_dense[(size_t)i * K + h->col[e2]] += h->val[e2];
+  }
+  delete h;
+  return NB_OK;
+}
+
+int nb_get_stats(const nb_ctx *c, int64_t *sum_finished, double *algorithmic_bytes, int64_t *kernel_launches) {
+  if (!c) return NB_ERR_ARG;
+  if (sum_finished) *sum_finished = c->sum_finished;
+  if (algorithmic_bytes) *algorithmic_bytes = c->alg_bytes;
+  if (kernel_launches) *kernel_launches = c->launches;
+  return NB_OK;
+}
+
+}  // extern "C"

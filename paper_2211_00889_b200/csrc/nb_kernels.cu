@@ -1,0 +1,382 @@
+// CUDA kernels (sm_100a) of the Non-blocking SGD aggregate-and-update step.
+//
+// Work decomposition: every thread owns 4 consecutive parameter columns for ALL K learners, every
+// CTA owns a contiguous column tile.  Nothing couples columns (the method only couples learners
+// and mini-batches), so CTAs never communicate, nothing waits on another CTA, and every output
+// element has exactly one writer.  All traffic is 128-bit (fp32) or 64-bit (bf16) per thread and
+// contiguous across a warp.  Gradient rows m >= n_i are never touched: skipping the abandoned
+// mini-batches is the method (Alg. 1: "break and abandon unfinished mini-batches").
+//
+// fp32 arithmetic is written with explicit round-to-nearest intrinsics so that the fused kernel
+// and the accumulate -> step pair perform the identical operation sequence and agree bit for bit.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "nb_internal.h"
+#include "nb_kernels.h"
+
+namespace nb {
+namespace {
+
+constexpr int kColsPerThread = 4;
+constexpr int kChunk = 8;  // gradient rows loaded back to back before they are summed
+
+__device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+
+// Raw 4-column gradient fragment as loaded, before widening.
+template <int SRC> struct Raw;
+template <> struct Raw<kSrcF32> { float4 r; };
+template <> struct Raw<kSrcBF16> { uint2 r; };
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+__device__ __forceinline__ float4 widen(const Raw<kSrcF32> &x) { return x.r; }
+__device__ __forceinline__ float4 widen(const Raw<kSrcBF16> &x) {
+  return make_float4(bf16_lo(x.r.x), bf16_hi(x.r.x), bf16_lo(x.r.y), bf16_hi(x.r.y));
+}
+
+// Loads columns [off, off+nvalid) of one gradient row; invalid lanes read as +0.  Streaming loads:
+// the gradient stream is read exactly once per step.
+template <bool ALIGNED>
+__device__ __forceinline__ Raw<kSrcF32> load_raw(const float *p, int nvalid, Raw<kSrcF32> *) {
+  Raw<kSrcF32> out;
+  if (ALIGNED && nvalid == 4) {
+    out.r = __ldcs(reinterpret_cast<const float4 *>(p));
+  } else {
+    out.r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (nvalid > 0) out.r.x = __ldcs(p);
+    if (nvalid > 1) out.r.y = __ldcs(p + 1);
+    if (nvalid > 2) out.r.z = __ldcs(p + 2);
+    if (nvalid > 3) out.r.w = __ldcs(p + 3);
+  }
+  return out;
+}
+template <bool ALIGNED>
+__device__ __forceinline__ Raw<kSrcBF16> load_raw(const uint16_t *p, int nvalid, Raw<kSrcBF16> *) {
+  Raw<kSrcBF16> out;
+  if (ALIGNED && nvalid == 4) {
+    out.r = __ldcs(reinterpret_cast<const uint2 *>(p));
+  } else {
+    uint32_t e0 = 0, e1 = 0, e2 = 0, e3 = 0;
+    if (nvalid > 0) e0 = __ldcs(p);
+    if (nvalid > 1) e1 = __ldcs(p + 1);
+    if (nvalid > 2) e2 = __ldcs(p + 2);
+    if (nvalid > 3) e3 = __ldcs(p + 3);
+    out.r = make_uint2(e0 | (e1 << 16), e2 | (e3 << 16));
+  }
+  return out;
+}
+
+template <int SRC> struct ElemOf;
+template <> struct ElemOf<kSrcF32> { using type = float; };
+template <> struct ElemOf<kSrcBF16> { using type = uint16_t; };
+
+// acc_i = sum_{m < n_i} G[i, m, cols], fp32, m ascending, starting from +0
+// (Alg. 1 accumulate step; Eq. 19).  SRC = kSrcAcc reads what nb_accumulate stored instead.
+template <int SRC, bool ALIGNED>
+__device__ __forceinline__ float4 gather(const StepArgs &a, int i, int64_t col0, int nvalid) {
+  if constexpr (SRC == kSrcAcc) {
+    return __ldcs(reinterpret_cast<const float4 *>(a.acc + (int64_t)i * a.ldx + col0));
+  } else {
+    using E = typename ElemOf<SRC>::type;
+    const E *base = reinterpret_cast<const E *>(a.G) + (int64_t)i * a.ld_k + col0;
+    const int n = a.n[i];
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int m0 = 0; m0 < n; m0 += kChunk) {
+      Raw<SRC> r[kChunk];
+#pragma unroll
+      for (int u = 0; u < kChunk; ++u)
+        if (m0 + u < n) r[u] = load_raw<ALIGNED>(base + (int64_t)(m0 + u) * a.ld_m, nvalid, (Raw<SRC> *)nullptr);
+#pragma unroll
+      for (int u = 0; u < kChunk; ++u)
+        if (m0 + u < n) {
+          const float4 g = widen(r[u]);
+          acc.x = __fadd_rn(acc.x, g.x);
+          acc.y = __fadd_rn(acc.y, g.y);
+          acc.z = __fadd_rn(acc.z, g.z);
+          acc.w = __fadd_rn(acc.w, g.w);
+        }
+    }
+    return acc;
+  }
+}
+
+// v' = mom * v + s * acc  (momentum; s is the per-learner normalisation / learning-rate adjustment)
+__device__ __forceinline__ float4 momentum(float mom, float4 v, float s, float4 g) {
+  return make_float4(__fmaf_rn(mom, v.x, __fmul_rn(s, g.x)), __fmaf_rn(mom, v.y, __fmul_rn(s, g.y)),
+                     __fmaf_rn(mom, v.z, __fmul_rn(s, g.z)), __fmaf_rn(mom, v.w, __fmul_rn(s, g.w)));
+}
+// x - lr * v
+__device__ __forceinline__ float4 descend(float4 x, float lr, float4 v) {
+  return make_float4(__fmaf_rn(-lr, v.x, x.x), __fmaf_rn(-lr, v.y, x.y), __fmaf_rn(-lr, v.z, x.z),
+                     __fmaf_rn(-lr, v.w, x.w));
+}
+__device__ __forceinline__ float4 add4(float4 a, float4 b) {
+  return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
+}
+__device__ __forceinline__ float4 scale4(float4 a, float s) {
+  return make_float4(__fmul_rn(a.x, s), __fmul_rn(a.y, s), __fmul_rn(a.z, s), __fmul_rn(a.w, s));
+}
+
+// sum_j W_ij x_j over the non-zeros of row i (Alg. 2 averaging step), from the staged tiles.
+__device__ __forceinline__ float4 mix_row(const float4 *xs, int tpb, int tid, const int32_t *s_col,
+                                          const float *s_val, int beg, int end) {
+  float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int e = beg; e < end; ++e) {
+    const float w = s_val[e];
+    const float4 x = xs[s_col[e] * tpb + tid];
+    r.x = __fmaf_rn(w, x.x, r.x);
+    r.y = __fmaf_rn(w, x.y, r.y);
+    r.z = __fmaf_rn(w, x.z, r.z);
+    r.w = __fmaf_rn(w, x.w, r.w);
+  }
+  return r;
+}
+
+// -------------------------------------------------------------------------------------------------
+// K1: masked accumulate.  grid = (column tiles, K)
+// -------------------------------------------------------------------------------------------------
+template <int SRC, bool ALIGNED>
+__global__ void __launch_bounds__(256) nb_accumulate_kernel(const __grid_constant__ StepArgs a) {
+  const int64_t col0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * kColsPerThread;
+  if (col0 >= a.P) return;
+  const int nvalid = (a.P - col0 < 4) ? (int)(a.P - col0) : 4;
+  const int i = blockIdx.y;
+  const float4 g = gather<SRC, ALIGNED>(a, i, col0, nvalid);
+  st4(a.acc + (int64_t)i * a.ldx + col0, g);
+}
+
+// -------------------------------------------------------------------------------------------------
+// K2 / K2f: normalise + momentum + mix + update (SRC = kSrcAcc), or the same fused with the masked
+// accumulate (SRC = kSrcF32 / kSrcBF16).
+//   MEAN = true : W = (1/K) 1 1^T; one column mean, no staging (Eq. 4-5).
+//   MEAN = false: sparse W; the thread's K old models are staged in shared memory so that row i can
+//                 pick its neighbours by index while X is updated in place (Alg. 2; Eq. 6).
+// -------------------------------------------------------------------------------------------------
+template <int SRC, bool ALIGNED, bool MEAN>
+__global__ void __launch_bounds__(256) nb_step_kernel(const __grid_constant__ StepArgs a) {
+  extern __shared__ float4 smem[];
+  const int tid = threadIdx.x;
+  const int tpb = blockDim.x;
+  const int K = a.K;
+  float4 *xs = smem;
+  int32_t *s_col = nullptr, *s_beg = nullptr, *s_end = nullptr;
+  float *s_val = nullptr;
+  if constexpr (!MEAN) {
+    s_col = reinterpret_cast<int32_t *>(smem + (size_t)K * tpb);
+    s_val = reinterpret_cast<float *>(s_col + a.mix_slots);
+    s_beg = reinterpret_cast<int32_t *>(s_val + a.mix_slots);
+    s_end = s_beg + K;
+    for (int e = tid; e < a.mix_slots; e += tpb) {
+      s_col[e] = a.mix->col[e];
+      s_val[e] = a.mix->val[e];
+    }
+    for (int e = tid; e < K; e += tpb) {
+      s_beg[e] = a.mix->row_beg[e];
+      s_end[e] = a.mix->row_end[e];
+    }
+    __syncthreads();
+  }
+  const int64_t col0 = ((int64_t)blockIdx.x * tpb + tid) * kColsPerThread;
+  if (col0 >= a.P) return;
+  const int nvalid = (a.P - col0 < 4) ? (int)(a.P - col0) : 4;
+  float *Xc = a.X + col0;
+  float *Vc = a.V + col0;
+  const int64_t ldx = a.ldx;
+  const float lr = a.lr, mom = a.mom;
+
+  if (a.order == NB_ORDER_MIX_THEN_UPDATE) {
+    float4 mean = make_float4(0.f, 0.f, 0.f, 0.f);
+    if constexpr (MEAN) {
+      for (int j = 0; j < K; ++j) mean = add4(mean, ld4(Xc + (int64_t)j * ldx));
+      mean = scale4(mean, a.inv_K);
+    } else {
+      for (int j = 0; j < K; ++j) xs[j * tpb + tid] = ld4(Xc + (int64_t)j * ldx);
+    }
+    for (int i = 0; i < K; ++i) {
+      const float4 v = ld4(Vc + (int64_t)i * ldx);
+      const float4 g = gather<SRC, ALIGNED>(a, i, col0, nvalid);
+      const float4 vn = momentum(mom, v, a.s[i], g);
+      float4 xh;
+      if constexpr (MEAN) xh = mean;
+      else xh = mix_row(xs, tpb, tid, s_col, s_val, s_beg[i], s_end[i]);
+      st4(Vc + (int64_t)i * ldx, vn);
+      st4(Xc + (int64_t)i * ldx, descend(xh, lr, vn));
+    }
+  } else {  // NB_ORDER_UPDATE_THEN_MIX: local step first, then average (Eq. 4-6)
+    float4 ysum = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < K; ++j) {
+      const float4 x = ld4(Xc + (int64_t)j * ldx);
+      const float4 v = ld4(Vc + (int64_t)j * ldx);
+      const float4 g = gather<SRC, ALIGNED>(a, j, col0, nvalid);
+      const float4 vn = momentum(mom, v, a.s[j], g);
+      st4(Vc + (int64_t)j * ldx, vn);
+      const float4 y = descend(x, lr, vn);
+      if constexpr (MEAN) ysum = add4(ysum, y);
+      else xs[j * tpb + tid] = y;
+    }
+    if constexpr (MEAN) {
+      const float4 m = scale4(ysum, a.inv_K);
+      for (int i = 0; i < K; ++i) st4(Xc + (int64_t)i * ldx, m);
+    } else {
+      for (int i = 0; i < K; ++i)
+        st4(Xc + (int64_t)i * ldx, mix_row(xs, tpb, tid, s_col, s_val, s_beg[i], s_end[i]));
+    }
+  }
+}
+
+// -------------------------------------------------------------------------------------------------
+// Non-blocking synchronous centralized step (Alg. 3): one shared model.
+//   g = (1/K) sum_i s_i acc_i ; v <- mom v + g ; x <- x - lr v
+// -------------------------------------------------------------------------------------------------
+template <int SRC, bool ALIGNED>
+__global__ void __launch_bounds__(256) nb_centralized_kernel(const __grid_constant__ StepArgs a) {
+  const int64_t col0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * kColsPerThread;
+  if (col0 >= a.P) return;
+  const int nvalid = (a.P - col0 < 4) ? (int)(a.P - col0) : 4;
+  float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int i = 0; i < a.K; ++i) {
+    const float4 g = gather<SRC, ALIGNED>(a, i, col0, nvalid);
+    const float s = a.s[i];
+    gs.x = __fmaf_rn(s, g.x, gs.x);
+    gs.y = __fmaf_rn(s, g.y, gs.y);
+    gs.z = __fmaf_rn(s, g.z, gs.z);
+    gs.w = __fmaf_rn(s, g.w, gs.w);
+  }
+  const float4 v = ld4(a.V + col0);
+  const float4 x = ld4(a.X + col0);
+  const float4 vn = momentum(a.mom, v, a.inv_K, gs);
+  st4(a.V + col0, vn);
+  st4(a.X + col0, descend(x, a.lr, vn));
+}
+
+// -------------------------------------------------------------------------------------------------
+// K3: MATCHA activation + W builder.  One Bernoulli draw per matching per step from the counter
+// generator; row i of W = I - alpha * sum_active L_j is written as (diagonal, active partners).
+// -------------------------------------------------------------------------------------------------
+__global__ void nb_matcha_build_kernel(const MatchaArgs a) {
+  const int i = threadIdx.x;
+  const uint32_t bits = matcha_bits(a.seed, a.step, a.n_matchings, a.thr);
+  const int stride = 1 + a.n_matchings;
+  if (i < a.K) {
+    const int e = i * stride;
+    int cnt = 0;
+    for (int c = 0; c < a.n_matchings; ++c) {
+      const int v = a.partner[c * a.K + i];
+      if (((bits >> c) & 1u) && v >= 0) {
+        ++cnt;
+        a.mix->col[e + cnt] = v;
+        a.mix->val[e + cnt] = a.alpha;
+      }
+    }
+    a.mix->col[e] = i;
+    a.mix->val[e] = __fsub_rn(1.0f, __fmul_rn(a.alpha, (float)cnt));
+    a.mix->row_beg[i] = e;
+    a.mix->row_end[i] = e + cnt + 1;
+  }
+  if (i == 0) {
+    a.mix->bits = bits;
+    a.mix->n_slots = a.K * stride;
+  }
+}
+
+// Average of the learners' models (Alg. 1 / Alg. 2 "Output"), ascending learner order.
+__global__ void __launch_bounds__(256) nb_mean_kernel(const float *X, int64_t ldx, int K, int64_t P, float *out) {
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= P) return;
+  float s = 0.f;
+  for (int i = 0; i < K; ++i) s = __fadd_rn(s, X[(int64_t)i * ldx + p]);
+  out[p] = __fdiv_rn(s, (float)K);
+}
+
+size_t step_smem_bytes(const StepArgs &a, int tpb) {
+  if (a.mean_mode) return 0;
+  return (size_t)a.K * tpb * sizeof(float4) + (size_t)a.mix_slots * 8 + (size_t)a.K * 8;
+}
+
+template <typename F> cudaError_t allow_big_smem(F *f) {
+  return cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+}
+
+template <int SRC, bool ALIGNED>
+cudaError_t launch_step_t(const StepArgs &a, cudaStream_t st) {
+  const int tpb = step_threads_per_block(a);
+  const int64_t per_block = (int64_t)tpb * kColsPerThread;
+  const unsigned grid = (unsigned)((a.P + per_block - 1) / per_block);
+  if (a.mean_mode)
+    nb_step_kernel<SRC, ALIGNED, true><<<grid, tpb, 0, st>>>(a);
+  else
+    nb_step_kernel<SRC, ALIGNED, false><<<grid, tpb, step_smem_bytes(a, tpb), st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int step_threads_per_block(const StepArgs &a) {
+  if (a.mean_mode) return 256;
+  // staged tile = K * threads * 16 B; keep several CTAs resident per SM
+  if (a.K <= 17) return 256;
+  if (a.K <= 35) return 128;
+  return 64;
+}
+
+cudaError_t configure_kernels() {
+  cudaError_t e;
+#define NB_CFG(SRC, AL) \
+  if ((e = allow_big_smem(nb_step_kernel<SRC, AL, false>)) != cudaSuccess) return e;
+  NB_CFG(kSrcF32, true) NB_CFG(kSrcF32, false) NB_CFG(kSrcBF16, true) NB_CFG(kSrcBF16, false)
+  NB_CFG(kSrcAcc, true)
+#undef NB_CFG
+  return cudaSuccess;
+}
+
+cudaError_t launch_accumulate(const StepArgs &a, int src, cudaStream_t st) {
+  const int tpb = 256;
+  const int64_t per_block = (int64_t)tpb * kColsPerThread;
+  dim3 grid((unsigned)((a.P + per_block - 1) / per_block), (unsigned)a.K);
+  if (src == kSrcF32) {
+    if (a.g_aligned) nb_accumulate_kernel<kSrcF32, true><<<grid, tpb, 0, st>>>(a);
+    else nb_accumulate_kernel<kSrcF32, false><<<grid, tpb, 0, st>>>(a);
+  } else {
+    if (a.g_aligned) nb_accumulate_kernel<kSrcBF16, true><<<grid, tpb, 0, st>>>(a);
+    else nb_accumulate_kernel<kSrcBF16, false><<<grid, tpb, 0, st>>>(a);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_step(const StepArgs &a, int src, cudaStream_t st) {
+  if (src == kSrcAcc) return launch_step_t<kSrcAcc, true>(a, st);
+  if (src == kSrcF32) return a.g_aligned ? launch_step_t<kSrcF32, true>(a, st) : launch_step_t<kSrcF32, false>(a, st);
+  return a.g_aligned ? launch_step_t<kSrcBF16, true>(a, st) : launch_step_t<kSrcBF16, false>(a, st);
+}
+
+cudaError_t launch_centralized(const StepArgs &a, int src, cudaStream_t st) {
+  const int tpb = 256;
+  const int64_t per_block = (int64_t)tpb * kColsPerThread;
+  const unsigned grid = (unsigned)((a.P + per_block - 1) / per_block);
+  if (src == kSrcAcc) nb_centralized_kernel<kSrcAcc, true><<<grid, tpb, 0, st>>>(a);
+  else if (src == kSrcF32) {
+    if (a.g_aligned) nb_centralized_kernel<kSrcF32, true><<<grid, tpb, 0, st>>>(a);
+    else nb_centralized_kernel<kSrcF32, false><<<grid, tpb, 0, st>>>(a);
+  } else {
+    if (a.g_aligned) nb_centralized_kernel<kSrcBF16, true><<<grid, tpb, 0, st>>>(a);
+    else nb_centralized_kernel<kSrcBF16, false><<<grid, tpb, 0, st>>>(a);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_matcha_build(const MatchaArgs &a, cudaStream_t st) {
+  nb_matcha_build_kernel<<<1, NB_MAX_K, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, cudaStream_t st) {
+  const unsigned grid = (unsigned)((P + 255) / 256);
+  nb_mean_kernel<<<grid, 256, 0, st>>>(X, ldx, K, P, out);
+  return cudaGetLastError();
+}
+
+}  // namespace nb

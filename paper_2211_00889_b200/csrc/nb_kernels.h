@@ -1,0 +1,60 @@
+// Device-side data structures and kernel launchers (internal).
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "nb.h"
+
+namespace nb {
+
+// Sparse mixing matrix in device memory.  Row i owns slots [row_beg[i], row_end[i]).  A fixed W is
+// uploaded once; the MATCHA builder kernel rewrites the table every step.
+struct MixTable {
+  int32_t row_beg[NB_MAX_K];
+  int32_t row_end[NB_MAX_K];
+  int32_t col[NB_MAX_NNZ];
+  float val[NB_MAX_NNZ];
+  uint32_t bits;      // MATCHA: activation word of the step the table was built for
+  int32_t n_slots;    // slots in use (upper bound of every row_end)
+  int32_t pad[2];
+};
+
+enum GradSource : int { kSrcF32 = 0, kSrcBF16 = 1, kSrcAcc = 2 };
+
+// Everything one step needs, passed by value as a kernel parameter (no per-step uploads).
+struct StepArgs {
+  float *X;            // [K, ldx] models (NB_CENTRALIZED: [1, ldx])
+  float *V;            // [K, ldx] momentum
+  float *acc;          // [K, ldx] accumulator (written by accumulate, read by the unfused step)
+  const void *G;       // gradient stream, element (i,m,p) at G[i*ld_k + m*ld_m + p]
+  const MixTable *mix; // sparse W (ignored in mean mode)
+  int64_t ldx, ld_m, ld_k, P;
+  int32_t K, M;
+  int32_t mix_slots;   // number of table slots to stage in shared memory
+  int32_t mean_mode;   // 1: W = (1/K) 1 1^T, computed as one column mean
+  int32_t order;       // nb_order
+  int32_t g_aligned;   // 1: G base, ld_m, ld_k allow 4-element vector loads
+  float lr, mom, inv_K;
+  int32_t n[NB_MAX_K]; // finished counts
+  float s[NB_MAX_K];   // per-learner scale (1/n_i or n_i/M)
+};
+
+struct MatchaArgs {
+  MixTable *mix;
+  const int32_t *partner;  // device [n_matchings*K]
+  uint64_t seed, thr;
+  int64_t step;
+  int32_t K, n_matchings;
+  float alpha;
+};
+
+int step_threads_per_block(const StepArgs &a);
+cudaError_t launch_accumulate(const StepArgs &a, int src, cudaStream_t st);
+cudaError_t launch_step(const StepArgs &a, int src, cudaStream_t st);
+cudaError_t launch_centralized(const StepArgs &a, int src, cudaStream_t st);
+cudaError_t launch_matcha_build(const MatchaArgs &a, cudaStream_t st);
+cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, cudaStream_t st);
+cudaError_t configure_kernels();
+
+}  // namespace nb

@@ -1,0 +1,52 @@
+"""The C-ABI library loads and exports every symbol include/nb.h declares (no compute calls)."""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    src = open(os.path.join(ROOT, "include", "nb.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    names = re.findall(r"\b(nb_[a-z_A-Z0-9]+)\s*\(", src)
+    return sorted(set(names))
+
+
+def test_header_declares_the_named_entry_points():
+    names = _declared()
+    for must in ("nb_create", "nb_accumulate", "nb_step", "nb_get_params", "nb_step_fused", "nb_destroy",
+                 "nb_straggler_sample", "nb_get_device_mixing"):
+        assert must in names
+
+
+def test_library_builds_loads_and_exports_every_declared_symbol():
+    from paper_2211_00889_b200.build import build_library
+    path = build_library()
+    lib = ctypes.CDLL(path)
+    for name in _declared():
+        assert hasattr(lib, name), name
+
+
+def test_binding_covers_every_declared_symbol():
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding
+    assert sorted(binding.EXPORTED) == _declared()
+
+
+def test_argument_errors_are_reported_without_a_gpu():
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    h = ctypes.c_void_p()
+    assert B.lib.nb_create(ctypes.byref(h), 0, 10, 1, 0.1, 0.9, B.NB_ALLREDUCE, None) == B.NB_ERR_ARG
+    assert b"K" in B.lib.nb_last_error(None)
+    assert B.lib.nb_create(ctypes.byref(h), 4, 0, 1, 0.1, 0.9, B.NB_ALLREDUCE, None) == B.NB_ERR_ARG
+    assert B.lib.nb_create(ctypes.byref(h), 4, 8, 0, 0.1, 0.9, B.NB_ALLREDUCE, None) == B.NB_ERR_ARG
+    assert B.lib.nb_create(ctypes.byref(h), 4, 8, 2, 0.1, 0.9, 9, None) == B.NB_ERR_ARG
+    assert B.lib.nb_create(ctypes.byref(h), 65, 8, 2, 0.1, 0.9, B.NB_ALLREDUCE, None) == B.NB_ERR_UNSUPPORTED
+    assert B.lib.nb_create(ctypes.byref(h), 4, 8, 2, 0.1, 0.9, B.NB_DPSGD, None) == B.NB_ERR_ARG   # needs a topology
+    assert h.value is None
+    assert B.lib.nb_destroy(None) == B.NB_OK
+    assert B.lib.nb_step(None, None) == B.NB_ERR_ARG

@@ -1,0 +1,137 @@
+"""Host logic of the library against the oracle, bit for bit: straggler simulator (finished counts,
+masks), random regular graph + matchings, MATCHA activation words, mixing matrices.  CPU only."""
+import numpy as np
+import pytest
+
+from oracle import nb_oracle as O
+from paper_2211_00889_b200.build import build_library
+
+build_library()
+from paper_2211_00889_b200 import binding as B  # noqa: E402
+from paper_2211_00889_b200.workloads import WORKLOADS  # noqa: E402
+
+
+@pytest.mark.parametrize("name", list(WORKLOADS))
+def test_finished_counts_and_masks_bit_exact(name):
+    w = WORKLOADS[name]
+    for t in range(300):
+        n, mask, tau = B.straggler_sample(w.straggler_model, w.seed, t, w.K, w.M, w.straggler_params)
+        want = O.straggler_counts(w.straggler_model, w.seed, t, w.K, w.M, w.straggler_params)
+        assert n.tolist() == want, (name, t)
+        assert np.array_equal(mask, O.finished_mask(want, w.M))
+        assert n.min() >= 1 and n.max() <= w.M
+        if w.straggler_model != "uniform_count":
+            assert n[int(np.argmin(tau))] == w.M
+
+
+def test_delays_bit_exact():
+    for t in range(200):
+        _, _, tau = B.straggler_sample("shifted_exp", 42, t, 16, 8, (1.0,))
+        assert tau.tolist() == O.delays_shifted_exp(42, t, 16, [1.0] * 16)
+
+
+def test_slow_set_bit_exact_through_delays():
+    K = 32
+    for t in range(200):
+        _, _, tau = B.straggler_sample("shifted_exp_slowset", 7, t, K, 8, (0.25, 2.0, 0.1))
+        slow = set(O.slow_set(7, t, K, 8))
+        want = O.delays_shifted_exp(7, t, K, [2.0 if i in slow else 0.1 for i in range(K)])
+        assert tau.tolist() == want
+
+
+def test_straggler_argument_errors():
+    import ctypes as C
+    cfg = B.nb_straggler()
+    n = np.zeros(4, dtype=np.int32)
+    p = n.ctypes.data_as(C.POINTER(C.c_int32))
+    cfg.model = 7
+    assert B.lib.nb_straggler_sample(C.byref(cfg), 4, 4, 0, p, None, None) == B.NB_ERR_ARG
+    cfg.model = B.NB_STRAG_SHIFTED_EXP
+    cfg.params[0] = -1.0
+    assert B.lib.nb_straggler_sample(C.byref(cfg), 4, 4, 0, p, None, None) == B.NB_ERR_ARG
+    cfg.params[0] = 1.0
+    assert B.lib.nb_straggler_sample(C.byref(cfg), 0, 4, 0, p, None, None) == B.NB_ERR_ARG
+    assert B.lib.nb_straggler_sample(C.byref(cfg), 4, 0, 0, p, None, None) == B.NB_ERR_ARG
+    assert B.lib.nb_straggler_sample(C.byref(cfg), 4, 4, 0, p, None, None) == B.NB_OK
+
+
+@pytest.mark.parametrize("seed,K,d", [(221100893, 16, 3), (1, 16, 3), (2, 8, 3), (3, 32, 3), (4, 10, 4), (5, 6, 5)])
+def test_random_regular_graph_and_matchings_bit_exact(seed, K, d):
+    topo, _ = B.make_topology("random_regular", degree=d, seed=seed, alpha=0.1, act_prob=0.5)
+    partner, attempts = B.topology_matchings(topo, K)
+    edges, want_attempts = O.random_regular_graph(seed, K, d)
+    want = O.greedy_matchings(edges, K)
+    assert attempts == want_attempts
+    assert partner.tolist() == want
+
+
+def test_matcha_activation_and_W_match_oracle():
+    w = WORKLOADS["cfg4_matcha_vgg16"]
+    topo, _ = B.make_topology("random_regular", degree=w.degree, seed=w.seed, alpha=w.alpha, act_prob=w.act_prob)
+    partner, _ = B.topology_matchings(topo, w.K)
+    for t in range(500):
+        W, bits = B.mixing_matrix(topo, B.NB_MATCHA, w.K, t)
+        want_bits = O.matcha_activation(w.seed, t, len(partner), w.act_prob)
+        assert bits == want_bits
+        Wd = O.matcha_W(partner.tolist(), want_bits, w.alpha, w.K)
+        assert np.abs(W.astype(np.float64) - Wd).max() < 1e-7
+        assert np.array_equal(W != 0, Wd != 0)
+
+
+@pytest.mark.parametrize("prob", [0.0, 1.0, 0.25, 0.9])
+def test_activation_probability_extremes(prob):
+    partner = np.array([[1, 0, 3, 2], [2, 3, 0, 1], [3, 2, 1, 0]], dtype=np.int32)
+    topo, _ = B.make_topology("matchings", partner=partner, seed=99, alpha=0.25, act_prob=prob)
+    for t in range(200):
+        _, bits = B.mixing_matrix(topo, B.NB_MATCHA, 4, t)
+        assert bits == O.matcha_activation(99, t, 3, prob)
+        if prob == 0.0:
+            assert bits == 0
+        if prob == 1.0:
+            assert bits == 0b111
+
+
+def test_fixed_mixing_matrices_match_oracle():
+    for K in (1, 2, 3, 16, 32):
+        topo, _ = B.make_topology("ring")
+        W, _ = B.mixing_matrix(topo, B.NB_DPSGD, K, 0)
+        assert np.abs(W.astype(np.float64) - O.ring_W(K)).max() < 1e-7
+        W, _ = B.mixing_matrix(None, B.NB_ALLREDUCE, K, 0)
+        assert np.array_equal(W.astype(np.float64), O.full_W(K))
+
+
+def test_topology_validation():
+    import ctypes as C
+    W = np.zeros((4, 4), dtype=np.float32)
+    Wp = W.ctypes.data_as(C.POINTER(C.c_float))
+    # CSR whose rows do not sum to one
+    topo, keep = B.make_topology("csr", csr=([0, 1, 2, 3, 4], [0, 1, 2, 3], [1.0, 1.0, 0.5, 1.0]))
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_DPSGD, 4, 0, Wp, None) == B.NB_ERR_ARG
+    # a good CSR (unsorted columns are accepted and sorted)
+    topo, keep = B.make_topology("csr", csr=([0, 2, 4, 5, 6], [1, 0, 0, 1, 2, 3], [0.25, 0.75, 0.25, 0.75, 1.0, 1.0]))
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_DPSGD, 4, 0, Wp, None) == B.NB_OK
+    assert W.tolist() == [[0.75, 0.25, 0, 0], [0.25, 0.75, 0, 0], [0, 0, 1, 0], [0, 0, 0, 1]]
+    # partner table that is not an involution
+    topo, keep = B.make_topology("matchings", partner=np.array([[1, 2, 0, -1]]), alpha=0.1, act_prob=0.5)
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_MATCHA, 4, 0, Wp, None) == B.NB_ERR_ARG
+    # edge repeated in two matchings
+    topo, keep = B.make_topology("matchings", partner=np.array([[1, 0, -1, -1], [1, 0, 3, 2]]), alpha=0.1, act_prob=0.5)
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_MATCHA, 4, 0, Wp, None) == B.NB_ERR_ARG
+    # alpha too large for the degree
+    topo, keep = B.make_topology("matchings", partner=np.array([[1, 0, 3, 2], [2, 3, 0, 1]]), alpha=0.6, act_prob=0.5)
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_MATCHA, 4, 0, Wp, None) == B.NB_ERR_ARG
+    # impossible regular graph (odd K*d)
+    topo, keep = B.make_topology("random_regular", degree=3, seed=1, alpha=0.1, act_prob=0.5)
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_MATCHA, 5, 0, Wp, None) == B.NB_ERR_ARG
+    # wrong topology for the variant
+    topo, keep = B.make_topology("ring")
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_MATCHA, 4, 0, Wp, None) == B.NB_ERR_ARG
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_ALLREDUCE, 4, 0, Wp, None) == B.NB_ERR_ARG
+
+
+def test_expected_finished_fraction_of_the_bench_workload():
+    # documents the size of the timed workload: mean of sum n_i over many steps
+    w = WORKLOADS["cfg3_dpsgd_ring_resnet50"]
+    tot = sum(int(B.straggler_sample(w.straggler_model, w.seed, t, w.K, w.M, w.straggler_params)[0].sum())
+              for t in range(3000))
+    assert 70.0 < tot / 3000 < 77.0
