@@ -108,18 +108,19 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
     return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
-def gradients_np(w: Workload, step: int):
+def gradients_np(w: Workload, step: int, with_unrounded: bool = False):
     """One step's mini-batch gradient stream G[K, M, P] drawn on the CPU.
 
     Returns (payload, values): `payload` is the array handed to the library (float32, or uint16
     bf16 storage bits); `values` is a float32 array holding exactly the numbers the payload
-    denotes (what the oracle consumes)."""
+    denotes (what the oracle consumes).  with_unrounded adds the fp32 draws before bf16 rounding."""
     g = _np_rng(w.seed, 1, step)
     a = g.standard_normal((w.K, w.M, w.P), dtype=np.float32) * np.float32(w.grad_sigma)
     if w.grad_dtype == "f32":
-        return a, a
+        return (a, a, a) if with_unrounded else (a, a)
     bits = round_to_bf16_bits(a)
-    return bits, bf16_bits_to_f32(bits)
+    vals = bf16_bits_to_f32(bits)
+    return (bits, vals, a) if with_unrounded else (bits, vals)
 
 
 def gradients_torch(w: Workload, step: int, device):

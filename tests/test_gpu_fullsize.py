@@ -1,0 +1,74 @@
+"""Parity at the full sizes of the named configurations, in the launch configuration bench.py
+times (dense, aligned gradient stream resident in HBM; nb_step_fused): the computation is
+independent per column, so the oracle recomputes a fixed set of column windows exactly - the first
+and last tiles, windows across tile boundaries and random windows - from the same input values."""
+import numpy as np
+import pytest
+
+from oracle import nb_oracle as O
+from paper_2211_00889_b200 import workloads as WL
+from tests import _harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _windows(P, rng, n_random=24, width=48):
+    wins = [(0, min(P, 1040)), (max(0, P - 1040), P)]
+    for t in (1, 2, 1000):                                   # straddle 1024-column tile boundaries
+        c = t * 1024
+        if c + 8 < P:
+            wins.append((c - 8, c + 8))
+    for _ in range(n_random):
+        c = int(rng.integers(0, max(1, P - width)))
+        wins.append((c, min(P, c + width)))
+    cols = np.unique(np.concatenate([np.arange(a, b) for a, b in wins]))
+    return cols
+
+
+@pytest.mark.parametrize("name,steps", [
+    ("cfg2_allreduce_resnet18", 10),
+    ("cfg3_dpsgd_ring_resnet50", 10),
+    ("cfg4_matcha_vgg16", 4),
+    ("cfg5_scale_allreduce", 2),
+    ("cfg5_scale_ring", 2),
+])
+def test_full_size_sampled_columns(name, steps):
+    import torch
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    w = WL.WORKLOADS[name]
+    es = 4 if w.grad_dtype == "f32" else 2
+    need = w.K * w.M * w.P * es + 4 * w.K * w.P * 4 + w.M * w.P * 4 + (2 << 30)
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < need:
+        pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
+    cols = _windows(w.P, np.random.default_rng(w.seed))
+    cols_dev = torch.from_numpy(cols).cuda()
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed)
+    x0 = torch.randn(w.P, generator=gen, device="cuda", dtype=torch.float32) * w.init_sigma
+    ctx = B.context_for(w)
+    ctx.set_params(x0)
+    orc = H.oracle_for(w, len(cols))
+    orc.set_params(x0[cols_dev].cpu().numpy())
+    del x0
+    for t in range(steps):
+        n = H.lib_counts(B, w, t)
+        G = WL.gradients_torch(w, t, "cuda")
+        ctx.step_fused(G, n)
+        Gs = G[:, :, cols_dev].float().cpu().numpy()          # exact values of the sampled columns
+        torch.cuda.synchronize()
+        del G
+        orc.step(Gs, n.tolist())
+        if w.variant == "matcha":
+            bits, Wdev = ctx.get_device_mixing()
+            assert bits == O.matcha_activation(w.seed, t, len(orc.partner), w.act_prob)
+    torch.cuda.empty_cache()
+    X = ctx.get_params(device="cuda")[:, cols_dev].cpu().numpy()
+    V = ctx.get_momentum(device="cuda")[:, cols_dev].cpu().numpy()
+    ctx.close()
+    torch.cuda.empty_cache()
+    H.assert_close(X, orc.X, H.TOL_SAME_INPUT, name + " X")
+    H.assert_close(V, orc.V, H.TOL_SAME_INPUT, name + " V")

@@ -1,0 +1,380 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the same
+seeded inputs.  Bit-exact for finished counts, masks and MATCHA activations; norm-wise 1e-5 on
+parameters against the oracle fed the same input values; 2e-3 for bf16 gradient inputs against
+the oracle fed the un-rounded fp32 gradients."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from oracle import nb_oracle as O
+from paper_2211_00889_b200 import workloads as WL
+from tests import _harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding
+    return binding
+
+
+def _run(B, w, steps, fused=True, norm="mean", order="mix_then_update", check_steps=(10,), with_unrounded=False,
+         pad=0):
+    """Runs library and oracle side by side; returns per-check-step errors."""
+    import torch
+    ctx = B.context_for(w)
+    ctx.set_option(B.NB_OPT_NORM, B.NB_NORM_MEAN if norm == "mean" else B.NB_NORM_PAPER)
+    ctx.set_option(B.NB_OPT_ORDER, B.NB_ORDER_MIX_THEN_UPDATE if order == "mix_then_update" else B.NB_ORDER_UPDATE_THEN_MIX)
+    orc = H.oracle_for(w, w.P, norm, order)
+    orc_unr = H.oracle_for(w, w.P, norm, order) if with_unrounded else None
+    x0 = WL.init_params(w)
+    ctx.set_params(torch.from_numpy(x0).cuda())
+    orc.set_params(x0)
+    if orc_unr:
+        orc_unr.set_params(x0)
+    out = {}
+    for t in range(steps):
+        n = H.lib_counts(B, w, t)
+        payload, values, unr = WL.gradients_np(w, t, with_unrounded=True)
+        if pad:
+            buf = np.zeros((w.K, w.M, w.P + pad), dtype=payload.dtype)
+            buf[:, :, :w.P] = payload
+            g = H.to_device(buf)
+            ld = dict(ld_m=w.P + pad, ld_k=w.M * (w.P + pad))
+        else:
+            g = H.to_device(payload)
+            ld = {}
+        if fused:
+            ctx.step_fused(g, n, **ld)
+        else:
+            ctx.accumulate(g, n, **ld)
+            ctx.step()
+        orc.step(values, n.tolist())
+        if orc_unr:
+            orc_unr.step(unr, n.tolist())
+        if w.variant == "matcha":
+            bits, Wdev = ctx.get_device_mixing()
+            want = O.matcha_activation(w.seed, t, len(orc.partner), w.act_prob)
+            assert bits == want == ctx.get_matcha_activation(t)          # bit-exact activation word
+            assert np.array_equal(Wdev, ctx.get_W(t))                     # device builder == host builder
+            assert np.abs(Wdev - O.matcha_W(orc.partner, want, w.alpha, w.K)).max() < 1e-7
+        if (t + 1) in check_steps or t == steps - 1:
+            X = ctx.get_params().numpy()
+            V = ctx.get_momentum().numpy()
+            e = H.assert_close(X, orc.X, H.TOL_SAME_INPUT, "%s step %d X" % (w.name, t + 1))
+            H.assert_close(V, orc.V, H.TOL_SAME_INPUT, "%s step %d V" % (w.name, t + 1))
+            H.assert_close(ctx.get_mean_params().numpy(), O.mean_params(orc.X), H.TOL_SAME_INPUT, "mean model")
+            if orc_unr:
+                H.assert_close(X, orc_unr.X, H.TOL_BF16_ROUNDING, "%s step %d X vs un-rounded" % (w.name, t + 1))
+            out[t + 1] = e
+    assert ctx.get_step() == steps
+    ctx.close()
+    return out
+
+
+# ----------------------------------------------------------------------------------------------
+# The five configurations, at sizes the oracle finishes in seconds that span several column
+# tiles and a ragged tail (cfg1 is run at its real size).
+# ----------------------------------------------------------------------------------------------
+def test_cfg1_tiny_allreduce_exact_size(B):
+    w = WL.WORKLOADS["cfg1_tiny_allreduce"]
+    _run(B, w, w.steps, fused=True)
+    _run(B, w, w.steps, fused=False)
+
+
+@pytest.mark.parametrize("name,P", [
+    ("cfg2_allreduce_resnet18", 5 * 1024 + 260),
+    ("cfg3_dpsgd_ring_resnet50", 4 * 1024 + 520),
+    ("cfg4_matcha_vgg16", 3 * 1024 + 8),
+    ("cfg5_scale_allreduce", 2 * 1024 + 36),
+    ("cfg5_scale_ring", 2 * 1024 + 36),
+])
+@pytest.mark.parametrize("fused", [True, False])
+def test_configs_scaled_columns(B, name, P, fused):
+    w = WL.scaled(WL.WORKLOADS[name], P, steps=12)
+    _run(B, w, w.steps, fused=fused, check_steps=(10,), with_unrounded=(w.grad_dtype == "bf16"))
+
+
+@pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16"])
+@pytest.mark.parametrize("P", [1, 3, 7, 4099, 1025])
+def test_ragged_and_unaligned_sizes(B, name, P):
+    # P not a multiple of 4: rows of the dense stream are not 16-byte aligned -> scalar-load kernels
+    w = WL.scaled(WL.WORKLOADS[name], P, steps=4)
+    _run(B, w, w.steps, fused=True)
+    _run(B, w, w.steps, fused=False)
+
+
+@pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50"])
+def test_padded_rows_take_the_vector_path_with_a_partial_last_vector(B, name):
+    # P = 4099 with row pitch 4104: aligned rows, last vector has 3 valid columns
+    w = WL.scaled(WL.WORKLOADS[name], 4099, steps=3)
+    _run(B, w, w.steps, fused=True, pad=5)
+    _run(B, w, w.steps, fused=False, pad=5)
+
+
+@pytest.mark.parametrize("name", ["cfg1_tiny_allreduce", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16"])
+@pytest.mark.parametrize("norm,order", [("paper", "mix_then_update"), ("mean", "update_then_mix"),
+                                        ("paper", "update_then_mix")])
+def test_norm_and_order_options(B, name, norm, order):
+    w = WL.scaled(WL.WORKLOADS[name], 2 * 1024 + 100, steps=6)
+    _run(B, w, w.steps, fused=True, norm=norm, order=order)
+    _run(B, w, w.steps, fused=False, norm=norm, order=order)
+
+
+# ----------------------------------------------------------------------------------------------
+# Self-consistency of the CUDA path (bitwise)
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16",
+                                  "cfg5_scale_ring"])
+def test_fused_equals_unfused_bitwise(B, name):
+    import torch
+    w = WL.scaled(WL.WORKLOADS[name], 3 * 1024 + 404, steps=5)
+    a, b = B.context_for(w), B.context_for(w)
+    x0 = torch.from_numpy(WL.init_params(w)).cuda()
+    a.set_params(x0)
+    b.set_params(x0)
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        g = H.to_device(WL.gradients_np(w, t)[0])
+        a.step_fused(g, n)
+        b.accumulate(g, n)
+        b.step()
+    assert torch.equal(a.get_params(), b.get_params())
+    assert torch.equal(a.get_momentum(), b.get_momentum())
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("name", ["cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16", "cfg2_allreduce_resnet18"])
+def test_column_subset_equals_full_run_bitwise(B, name):
+    """Columns never interact: running a column slice alone gives the same bits as the full run."""
+    import torch
+    P, c0, c1 = 4 * 1024 + 96, 1024 + 8, 3 * 1024 + 40
+    w = WL.scaled(WL.WORKLOADS[name], P, steps=4)
+    ws = replace(w, P=c1 - c0)
+    full, part = B.context_for(w), B.context_for(ws)
+    x0 = WL.init_params(w)
+    full.set_params(torch.from_numpy(x0).cuda())
+    part.set_params(torch.from_numpy(x0[c0:c1].copy()).cuda())
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        payload = WL.gradients_np(w, t)[0]
+        full.step_fused(H.to_device(payload), n)
+        part.step_fused(H.to_device(payload[:, :, c0:c1]), n)
+    assert torch.equal(full.get_params()[:, c0:c1], part.get_params())
+    full.close(); part.close()
+
+
+def test_strided_view_of_a_wider_stream_equals_dense(B):
+    """ld_m / ld_k: a column window of a wider gradient buffer, addressed in place."""
+    import torch
+    P, c0, c1 = 3 * 1024, 512, 2 * 1024 + 512
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], P, steps=3)
+    ws = replace(w, P=c1 - c0)
+    a, b = B.context_for(ws), B.context_for(ws)
+    x0 = torch.from_numpy(WL.init_params(ws)).cuda()
+    a.set_params(x0); b.set_params(x0)
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        g = H.to_device(WL.gradients_np(w, t)[0])
+        view = g[:, :, c0:c1]                      # not contiguous
+        a.step_fused(view, n, ld_m=P, ld_k=w.M * P)
+        b.step_fused(view.contiguous(), n)
+    assert torch.equal(a.get_params(), b.get_params())
+    a.close(); b.close()
+
+
+def test_checkpoint_resume_is_bitwise(B):
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg4_matcha_vgg16"], 2 * 1024 + 12, steps=10)
+    x0 = torch.from_numpy(WL.init_params(w)).cuda()
+    straight = B.context_for(w)
+    straight.set_params(x0)
+    first = B.context_for(w)
+    first.set_params(x0)
+    for t in range(10):
+        n = H.lib_counts(B, w, t)
+        g = H.to_device(WL.gradients_np(w, t)[0])
+        straight.step_fused(g, n)
+        if t < 5:
+            first.step_fused(g, n)
+    X, V, step = first.get_params(), first.get_momentum(), first.get_step()
+    first.close()
+    second = B.context_for(w)
+    second.set_state(step, X, V)                     # host tensors in
+    for t in range(5, 10):
+        n = H.lib_counts(B, w, t)
+        second.step_fused(H.to_device(WL.gradients_np(w, t)[0]), n)
+    assert torch.equal(second.get_params(), straight.get_params())
+    assert torch.equal(second.get_momentum(), straight.get_momentum())
+    straight.close(); second.close()
+
+
+# ----------------------------------------------------------------------------------------------
+# Exact-arithmetic cases: every fp32 operation is exact, so GPU == oracle bit for bit
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("variant", ["allreduce", "dpsgd_identity", "matcha"])
+def test_exact_arithmetic_matches_oracle_bit_for_bit(B, variant):
+    import torch
+    K, P, M = 4, 1024 + 36, 4
+    lr, mom = 0.25, 0.5
+    rng = np.random.default_rng(17)
+    x0 = (rng.integers(-64, 65, P) / 4.0).astype(np.float32)
+    if variant == "allreduce":
+        ctx = B.NbContext(K, P, M, lr, mom, "allreduce")
+        orc = O.Oracle(K, P, M, lr, mom, "allreduce")
+    elif variant == "dpsgd_identity":
+        csr = (np.arange(K + 1), np.arange(K), np.ones(K))
+        ctx = B.NbContext(K, P, M, lr, mom, "dpsgd", B.make_topology("csr", csr=csr))
+        orc = O.Oracle(K, P, M, lr, mom, "dpsgd", W=O.identity_W(K))
+    else:
+        partner = [[1, 0, 3, 2], [2, 3, 0, 1]]
+        ctx = B.NbContext(K, P, M, lr, mom, "matcha",
+                          B.make_topology("matchings", partner=np.array(partner), seed=5, alpha=0.25, act_prob=0.5))
+        orc = O.Oracle(K, P, M, lr, mom, "matcha", partner=partner, alpha=0.25, prob=0.5, seed=5)
+    ctx.set_params(torch.from_numpy(x0).cuda())
+    orc.set_params(x0)
+    for t in range(3):
+        G = rng.integers(-8, 9, (K, M, P)).astype(np.float32)
+        n = [int(v) for v in rng.choice([1, 2, 4], K)]
+        ctx.step_fused(torch.from_numpy(G).cuda(), n)
+        orc.step(G, n)
+        X = ctx.get_params().numpy()
+        assert np.array_equal(X.astype(np.float64), orc.X), (variant, t)
+        assert np.array_equal(ctx.get_momentum().numpy().astype(np.float64), orc.V)
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------------------------
+# Degenerate cases and the other entry points
+# ----------------------------------------------------------------------------------------------
+def test_zero_finished_learner_and_single_learner(B):
+    import torch
+    # n_i = 0: no gradient contribution; momentum decays, mixing still happens
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 1024 + 4, steps=3)
+    w = replace(w, K=5)
+    ctx = B.context_for(w)
+    orc = H.oracle_for(w, w.P)
+    x0 = WL.init_params(w)
+    ctx.set_params(torch.from_numpy(x0).cuda()); orc.set_params(x0)
+    for t in range(3):
+        payload, values = WL.gradients_np(w, t)
+        n = [0, w.M, 1, 0, 3] if t != 1 else [0] * 5
+        ctx.step_fused(H.to_device(payload), n)
+        orc.step(values, n)
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+    ctx.close()
+    # K = 1, M = 1
+    w1 = replace(WL.scaled(WL.WORKLOADS["cfg2_allreduce_resnet18"], 77, steps=2), K=1, M=1)
+    ctx = B.context_for(w1); orc = H.oracle_for(w1, 77)
+    x0 = WL.init_params(w1)
+    ctx.set_params(torch.from_numpy(x0).cuda()); orc.set_params(x0)
+    for t in range(2):
+        payload, values = WL.gradients_np(w1, t)
+        ctx.step_fused(H.to_device(payload), [1]); orc.step(values, [1])
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+    ctx.close()
+
+
+def test_masked_accumulate_alone(B):
+    """nb_accumulate's output against the oracle's prefix sums; abandoned rows are never read
+    (they hold NaN here)."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 2 * 1024 + 24, steps=1)
+    ctx = B.context_for(w)
+    payload, values = WL.gradients_np(w, 0)
+    n = H.lib_counts(B, w, 0)
+    g = H.to_device(payload)
+    for i in range(w.K):
+        g[i, int(n[i]):] = float("nan")
+    ctx.accumulate(g, n)
+    acc = ctx.get_accumulator().numpy()
+    assert np.isfinite(acc).all()
+    H.assert_close(acc, O.accumulate(values, n.tolist()), 1e-6)
+    ctx.close()
+
+
+def test_per_learner_initialisation_and_large_k(B):
+    import torch
+    K, P, M = 40, 1024 + 8, 2
+    rng = np.random.default_rng(3)
+    X0 = rng.standard_normal((K, P)).astype(np.float32)
+    ctx = B.NbContext(K, P, M, 0.1, 0.9, "dpsgd", B.make_topology("ring"))
+    orc = O.Oracle(K, P, M, 0.1, 0.9, "dpsgd", W=O.ring_W(K))
+    ctx.set_params(torch.from_numpy(X0).cuda(), per_learner=True); orc.set_params(X0)
+    for t in range(3):
+        G = rng.standard_normal((K, M, P)).astype(np.float32)
+        n = rng.integers(0, M + 1, K).tolist()
+        ctx.step_fused(torch.from_numpy(G).cuda(), n); orc.step(G, n)
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+    ctx.close()
+
+
+def test_centralized_variant(B):
+    import torch
+    K, P, M = 8, 3 * 1024 + 5, 4
+    rng = np.random.default_rng(4)
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    for fused in (True, False):
+        ctx = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
+        ctx.set_params(torch.from_numpy(x0).cuda())
+        x, v = x0.astype(np.float64), np.zeros(P)
+        for t in range(6):
+            G = (np.random.default_rng(100 + t).standard_normal((K, M, P)) * 0.01).astype(np.float32)
+            n = np.random.default_rng(200 + t).integers(1, M + 1, K).tolist()
+            if fused:
+                ctx.step_fused(torch.from_numpy(G).cuda(), n)
+            else:
+                ctx.accumulate(torch.from_numpy(G).cuda(), n); ctx.step()
+            x, v = O.step_centralized(x, v, G, n, 0.1, 0.9)
+        H.assert_close(ctx.get_params().numpy(), x, H.TOL_SAME_INPUT)
+        H.assert_close(ctx.get_momentum().numpy(), v, H.TOL_SAME_INPUT)
+        H.assert_close(ctx.get_mean_params().numpy(), x, H.TOL_SAME_INPUT)
+        ctx.close()
+
+
+def test_host_buffer_entry_point(B):
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 2 * 1024 + 20, steps=3)
+    a, b = B.context_for(w), B.context_for(w)
+    x0 = torch.from_numpy(WL.init_params(w)).cuda()
+    a.set_params(x0); b.set_params(x0)
+    mean = torch.empty(w.P, dtype=torch.float32).pin_memory()
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        payload = WL.gradients_np(w, t)[0]
+        host = torch.from_numpy(payload).view(torch.bfloat16).pin_memory()
+        a.step_fused_host(host, n, mean_out=mean)
+        b.step_fused(H.to_device(payload), n)
+        assert torch.equal(mean, b.get_mean_params())
+    assert torch.equal(a.get_params(), b.get_params())
+    a.close(); b.close()
+
+
+def test_error_reporting(B):
+    import torch
+    ctx = B.NbContext(4, 100, 4, 0.1, 0.9, "allreduce")
+    with pytest.raises(B.NbError) as e:
+        ctx.step()
+    assert e.value.code == B.NB_ERR_STATE
+    g = torch.zeros((4, 4, 100), device="cuda")
+    with pytest.raises(B.NbError) as e:
+        ctx.step_fused(g, [1, 2, 5, 1])
+    assert e.value.code == B.NB_ERR_ARG
+    with pytest.raises(B.NbError):
+        ctx.step_fused(g, [1, 2, -1, 1])
+    with pytest.raises(B.NbError):
+        ctx.step_fused(g, [1, 1, 1, 1], ld_m=50)
+    ctx.accumulate(g, [1, 1, 1, 1])
+    ctx.step()
+    with pytest.raises(B.NbError):
+        ctx.step()                                   # accumulator already consumed
+    st = ctx.get_stats()
+    assert st["sum_finished"] == 4 and st["kernel_launches"] == 2
+    assert st["algorithmic_bytes"] == 100 * (4 * 4 + 16 * 4)
+    ctx.close()
