@@ -46,6 +46,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cols", type=int, default=0, help="profiling aid: run the workload on this many columns instead of its P")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -316,6 +317,9 @@ def main():
     args = parse_args()
     from paper_2211_00889_b200 import workloads as WL
     w = WL.WORKLOADS[args.workload]
+    if args.cols:
+        from dataclasses import replace
+        w = replace(WL.scaled(w, args.cols), name="%s[P=%d]" % (w.name, args.cols))
     if args.impl == "reference":
         run_reference(args, w)
     else:
