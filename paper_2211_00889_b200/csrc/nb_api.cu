@@ -20,6 +20,7 @@ struct nb_ctx {
   float *X = nullptr, *V = nullptr, *acc = nullptr, *d_mean = nullptr;
   nb::MixTable *d_mix = nullptr;
   int32_t *d_partner = nullptr;
+  int *d_err = nullptr;  // device word a kernel sets when one of its bounded waits runs out
   void *staging = nullptr;
   size_t staging_bytes = 0;
   int64_t step = 0;
@@ -164,14 +165,27 @@ int run_update(nb_ctx *c, nb::StepArgs *a, int src, cudaStream_t st) {
   fill_update_args(c, a);
   if (c->variant == NB_CENTRALIZED) {
     NB_CUDA(c, nb::launch_centralized(*a, src, st));
+    c->launches++;
   } else {
     int rc = build_device_mixing(c, st);
     if (rc != NB_OK) return rc;
-    NB_CUDA(c, nb::launch_step(*a, src, st));
+    int n_launched = 0;
+    cudaError_t e = nb::launch_step(*a, src, c->d_err, &n_launched, st);
+    c->launches += n_launched;
+    if (e != cudaSuccess) return cuda_fail(c, e, "launch_step");
   }
-  c->launches++;
   c->step++;
   c->acc_fresh = false;
+  return NB_OK;
+}
+
+// Reads the device error word (the stream is drained first).  A kernel sets it when one of its
+// bounded waits ran out; that is a defect, reported as a sticky NB_ERR_CUDA.
+int check_device_error(nb_ctx *c, cudaStream_t st) {
+  int h = 0;
+  NB_CUDA(c, cudaMemcpyAsync(&h, c->d_err, sizeof(int), cudaMemcpyDeviceToHost, st));
+  NB_CUDA(c, cudaStreamSynchronize(st));
+  if (h != 0) return fail(c, NB_ERR_CUDA, "device-side wait timed out (code " + std::to_string(h) + ")");
   return NB_OK;
 }
 
@@ -181,7 +195,7 @@ int copy_rows_out(nb_ctx *c, float *dst, const float *src, int rows, cudaStream_
   for (int r = 0; r < rows; ++r)
     NB_CUDA(c, cudaMemcpyAsync(dst + (int64_t)r * c->P, src + (int64_t)r * c->ldx, sizeof(float) * (size_t)c->P,
                                cudaMemcpyDefault, st));
-  if (!is_device_pointer(dst)) NB_CUDA(c, cudaStreamSynchronize(st));
+  if (!is_device_pointer(dst)) return check_device_error(c, st);
   return NB_OK;
 }
 int copy_rows_in(nb_ctx *c, float *dst, const float *src, int rows, cudaStream_t st) {
@@ -239,6 +253,8 @@ int nb_create(nb_ctx **out, int K, int64_t P, int M, float lr, float mom, int va
   if ((e = cudaMemset(c->X, 0, model_bytes)) != cudaSuccess) return bail(e, "cudaMemset(X)");
   if ((e = cudaMemset(c->V, 0, model_bytes)) != cudaSuccess) return bail(e, "cudaMemset(V)");
   if ((e = cudaMemset(c->acc, 0, acc_bytes)) != cudaSuccess) return bail(e, "cudaMemset(acc)");
+  if ((e = cudaMalloc(&c->d_err, sizeof(int))) != cudaSuccess) return bail(e, "cudaMalloc(err)");
+  if ((e = cudaMemset(c->d_err, 0, sizeof(int))) != cudaSuccess) return bail(e, "cudaMemset(err)");
   if (variant == NB_DPSGD || variant == NB_MATCHA) {
     if ((e = cudaMalloc(&c->d_mix, sizeof(nb::MixTable))) != cudaSuccess) return bail(e, "cudaMalloc(mix)");
     nb::MixTable *h = new (std::nothrow) nb::MixTable;
@@ -273,6 +289,7 @@ int nb_destroy(nb_ctx *c) {
   cudaFree(c->d_mean);
   cudaFree(c->d_mix);
   cudaFree(c->d_partner);
+  cudaFree(c->d_err);
   cudaFree(c->staging);
   cudaGetLastError();
   delete c;
@@ -402,8 +419,7 @@ int nb_step_fused_host(nb_ctx *c, const void *grads_host, int dtype, int64_t ld_
     rc = nb_get_mean_params(c, mean_out, stream);
     if (rc != NB_OK) return rc;
   }
-  NB_CUDA(c, cudaStreamSynchronize(st));
-  return NB_OK;
+  return check_device_error(c, st);
 }
 
 int nb_get_params(nb_ctx *c, float *dst, void *stream) {
@@ -435,7 +451,7 @@ int nb_get_mean_params(nb_ctx *c, float *dst, void *stream) {
   c->launches++;
   if (!dev) {
     NB_CUDA(c, cudaMemcpyAsync(dst, out, sizeof(float) * (size_t)c->P, cudaMemcpyDeviceToHost, st));
-    NB_CUDA(c, cudaStreamSynchronize(st));
+    return check_device_error(c, st);
   }
   return NB_OK;
 }

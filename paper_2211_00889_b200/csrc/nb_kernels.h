@@ -49,9 +49,27 @@ struct MatchaArgs {
   float alpha;
 };
 
+// Bulk-copy pipeline kernel (nb_pipeline.cu)
+struct PipeArgs {
+  StepArgs s;
+  int32_t T;              // columns per tile (multiple of 128)
+  int32_t n_slots;        // ring slots
+  int32_t rows_per_item;  // gradient rows per ring item
+  int32_t n_tiles;        // full tiles covered by the kernel
+  int *err;               // device word: 0, or the code of the wait that ran out
+};
+struct PipePlan {
+  int T, rows_per_item, n_slots, smem_bytes, n_tiles, grid;
+};
+bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan);
+cudaError_t configure_pipeline();
+cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan, int *err_flag, cudaStream_t st);
+
 int step_threads_per_block(const StepArgs &a);
 cudaError_t launch_accumulate(const StepArgs &a, int src, cudaStream_t st);
-cudaError_t launch_step(const StepArgs &a, int src, cudaStream_t st);
+// Runs the step on all P columns: pipeline kernel on the full tiles when it applies, direct-load
+// kernel on the rest.  *launches receives the number of kernels launched.
+cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st);
 cudaError_t launch_centralized(const StepArgs &a, int src, cudaStream_t st);
 cudaError_t launch_matcha_build(const MatchaArgs &a, cudaStream_t st);
 cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, cudaStream_t st);
