@@ -50,16 +50,8 @@ struct MatchaArgs {
 };
 
 // Bulk-copy pipeline kernel (nb_pipeline.cu)
-struct PipeArgs {
-  StepArgs s;
-  int32_t T;              // columns per tile (multiple of 128)
-  int32_t n_slots;        // ring slots
-  int32_t rows_per_item;  // gradient rows per ring item
-  int32_t n_tiles;        // full tiles covered by the kernel
-  int *err;               // device word: 0, or the code of the wait that ran out
-};
 struct PipePlan {
-  int T, rows_per_item, n_slots, smem_bytes, n_tiles, grid;
+  int T, rows_per_item, n_slots, n_groups, smem_bytes, n_tiles, grid;
 };
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan);
 cudaError_t configure_pipeline();

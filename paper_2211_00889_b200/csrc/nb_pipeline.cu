@@ -2,16 +2,18 @@
 //
 // The step is bound by HBM bandwidth, and what limits a plain load/store kernel is the number of
 // bytes it can keep in flight: every outstanding load pins registers of a resident thread.  Here
-// the loads are issued by ONE producer thread per CTA as 1-D bulk asynchronous copies
-// (cp.async.bulk, global -> shared, completion counted on an mbarrier), so the bytes in flight are
-// bounded by shared memory, not by occupancy:
+// the loads are issued by ONE producer thread per CTA as tiled bulk asynchronous copies (TMA:
+// cp.async.bulk.tensor through tensor maps, global -> shared, completion counted on an mbarrier),
+// so the bytes in flight are bounded by shared memory, not by occupancy, and one instruction moves
+// a whole box of rows (the producer is issue-bound with one instruction per row):
 //
 //   * the CTA owns column tiles of T columns (persistent, tile = blockIdx.x + k * gridDim.x);
-//   * per tile the producer first brings the K old model rows X[j, tile] into the X stage (the mix
-//     needs every neighbour's OLD value while X is updated in place), then streams, learner by
-//     learner, "items" into a ring of slots: item = momentum row V[i, tile] + up to R finished
-//     gradient rows G[i, m, tile]; rows m >= n_i are never requested (the abandoned mini-batches
-//     of Alg. 1 cost no bandwidth);
+//   * per tile the producer first brings the K old model rows X[:, tile] into the X stage with one
+//     box copy (the mix needs every neighbour's OLD value while X is updated in place), then
+//     streams, learner by learner, "items" into a ring of slots: item = momentum row V[i, tile]
+//     (one box) + up to R finished gradient rows G[i, m0:m0+r, tile] (one box of exactly r rows,
+//     from the tensor map whose box height is r); rows m >= n_i are never requested (the
+//     abandoned mini-batches of Alg. 1 cost no bandwidth);
 //   * T/4 consumer threads wait on a slot's "full" barrier, sum the rows in fp32 (m ascending),
 //     apply normalisation + momentum + mix + update with the same operation sequence as the
 //     direct-load kernels (bit-identical results), store x_i and v_i with 128-bit stores and hand
@@ -20,10 +22,12 @@
 // No CTA ever waits on another CTA.  Every mbarrier wait is bounded: after ~1 s of cycles a
 // waiting thread records an error code in global memory, all roles drain and the kernel returns
 // (the host reports it as an error status); nothing traps.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
 #include <cstdlib>
+#include <cstring>
 
 #include "nb_device.cuh"
 #include "nb_internal.h"
@@ -78,13 +82,21 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *e
   }
   return true;
 }
-// 1-D bulk copy global -> shared; completion is counted in bytes on `bar`.  dst, src and bytes are
-// multiples of 16.
-__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
+// Tiled bulk copies global -> shared through a tensor map; completion is counted in bytes on `bar`.
+// Coordinates are in map elements, innermost first; c0 * element size is a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
+      : "memory");
 }
 __device__ __forceinline__ void drain_and_exit_delay() {
   const long long t0 = clock64();
@@ -92,19 +104,36 @@ __device__ __forceinline__ void drain_and_exit_delay() {
   }
 }
 
+constexpr int kMaxRowsPerItem = 8;
+constexpr int kMaxGroups = 4;
+constexpr int kBoxInner = 256;  // a box is at most 256 elements wide: rows are described in units of T*es/256 bytes
+
+struct PipeArgs {
+  StepArgs s;
+  int32_t T;              // columns per tile (multiple of 128)
+  int32_t n_slots;        // ring slots
+  int32_t rows_per_item;  // gradient rows per ring item (R)
+  int32_t n_tiles;        // full tiles covered by the kernel
+  int32_t n_groups;       // consumer groups (each T/4 threads)
+  int *err;               // device word: 0, or the code of the wait that ran out
+  alignas(64) CUtensorMap xmap;                   // X as [K, units]: box = (256, K)
+  alignas(64) CUtensorMap vmap;                   // V as [K, units]: box = (256, 1)
+  alignas(64) CUtensorMap gmap[kMaxRowsPerItem];  // G as [K, M, units]: box = (256, r, 1), r = 1..R
+};
+
 struct PipeLayout {
   int32_t off_tab, off_xs, off_slots, slot_bytes, total;
 };
 
 __host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, int n_slots, int mix_slots) {
   PipeLayout L;
-  int off = (2 * n_slots + 2) * 8;
+  int off = (2 * n_slots + 5) * 8;
   off = (off + 127) / 128 * 128;
   L.off_tab = off;
   off += mix_slots * 8 + K * 8;
   off = (off + 127) / 128 * 128;
   L.off_xs = off;
-  off += K * T * 4;
+  off += 2 * K * T * 4;  // the X stage is double-buffered: tile t+1's models load while tile t is consumed
   L.off_slots = off;
   L.slot_bytes = T * 4 + R * T * es;
   L.total = off + n_slots * L.slot_bytes;
@@ -113,32 +142,38 @@ __host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, i
 
 // ES = bytes per gradient element (2: bf16, 4: fp32).
 template <int ES, bool MEAN>
-__global__ void __launch_bounds__(32 + 256, 2) nb_step_pipeline_kernel(const __grid_constant__ PipeArgs a) {
+__global__ void __launch_bounds__(32 + 512, 1) nb_step_pipeline_kernel(const __grid_constant__ PipeArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
   const StepArgs &s = a.s;
-  const int K = s.K, T = a.T, R = a.rows_per_item, NS = a.n_slots;
+  const int K = s.K, T = a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
+  const int NSG = NS / NG;  // slots in each group's ring
   const PipeLayout L = pipe_layout(K, T, ES, R, NS, s.mix_slots);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);
   uint64_t *empty = full + NS;
   uint64_t *xfull = empty + NS;
-  uint64_t *xempty = xfull + 1;
+  uint64_t *xempty = xfull + 2;
+  uint64_t *ybar = xfull + 4;
   int32_t *s_col = reinterpret_cast<int32_t *>(smem_raw + L.off_tab);
   float *s_val = reinterpret_cast<float *>(s_col + s.mix_slots);
   int32_t *s_beg = reinterpret_cast<int32_t *>(s_val + s.mix_slots);
   int32_t *s_end = s_beg + K;
-  float *xs = reinterpret_cast<float *>(smem_raw + L.off_xs);
+  float *xs_base = reinterpret_cast<float *>(smem_raw + L.off_xs);  // two stages of K*T floats
   unsigned char *slots = smem_raw + L.off_slots;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_cons_warps = T / 128;
+  const int group_warps = T / 128;                 // warps of one consumer group
+  const int n_cons_warps = group_warps * a.n_groups;
   if (threadIdx.x == 0) {
     for (int q = 0; q < NS; ++q) {
       mbar_init(&full[q], 1);
-      mbar_init(&empty[q], n_cons_warps);
+      mbar_init(&empty[q], group_warps);            // released by the group that owns the ring
     }
-    mbar_init(xfull, 1);
-    mbar_init(xempty, n_cons_warps);
+    for (int q = 0; q < 2; ++q) {
+      mbar_init(&xfull[q], 1);
+      mbar_init(&xempty[q], n_cons_warps);
+    }
+    mbar_init(ybar, n_cons_warps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if constexpr (!MEAN) {
@@ -159,67 +194,91 @@ __global__ void __launch_bounds__(32 + 256, 2) nb_step_pipeline_kernel(const __g
   if (warp == 0) {
     // ------------------------------------------------------------------ producer (one thread)
     if (lane == 0) {
-      const unsigned char *G = reinterpret_cast<const unsigned char *>(s.G);
-      uint32_t slot = 0, phase = 0;
+      // Every consumer group has a private ring of NSG slots (items of learner i go to ring i % NG):
+      // a slot is then always filled for, and released by, the same group, in order, which is
+      // what makes waiting on a phase parity unambiguous.
+      uint32_t ring_slot = 0;   // 8 bits per group: next slot of that group's ring
+      uint32_t ring_phase = 0;  // 1 bit per group: phase parity of that ring
       int titer = 0;
+      // X stage b = titer & 1 is reused every second tile; its k-th use waits for the (k-1)-th release
+      auto issue_x = [&](int tile_x, int it_x) -> bool {
+        const int b = it_x & 1;
+        if (!mbar_wait(&xempty[b], ((it_x >> 1) & 1) ^ 1, a.err, 1)) return false;
+        mbar_expect_tx(&xfull[b], (uint32_t)(K * T * 4));
+        tma_load_2d(xs_base + (size_t)b * K * T, &a.xmap, tile_x * kBoxInner, 0, &xfull[b]);
+        return true;
+      };
+      if (blockIdx.x < a.n_tiles) ok = issue_x(blockIdx.x, 0);
       for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x, ++titer) {
-        const int64_t col0 = (int64_t)tile * T;
-        if (!(ok = mbar_wait(xempty, (titer & 1) ^ 1, a.err, 1))) break;
-        mbar_expect_tx(xfull, (uint32_t)(K * T * 4));
-        for (int j = 0; j < K; ++j) bulk_load(xs + (size_t)j * T, s.X + (int64_t)j * ldx + col0, T * 4, xfull);
-        for (int i = 0; ok && i < K; ++i) {
+        const int c0 = tile * kBoxInner;  // the tile's first unit in every map
+        const bool have_next = tile + (int)gridDim.x < a.n_tiles;
+        int g = 0;  // i % NG
+        for (int i = 0; ok && i < K; ++i, g = (g + 1 == NG) ? 0 : g + 1) {
+          // the next tile's models are requested half-way through this tile: late enough that the
+          // stage they replace (tile t-1's) has been released, early enough to hide the latency
+          if (have_next && i == K / 2 && !(ok = issue_x(tile + gridDim.x, titer + 1))) break;
           const int n = s.n[i];
           int m0 = 0;
           do {
             const int rows = (n - m0 < R) ? (n - m0) : R;
-            if (!(ok = mbar_wait(&empty[slot], phase ^ 1, a.err, 2))) break;
-            unsigned char *dst = slots + (size_t)slot * L.slot_bytes;
+            const uint32_t gs = (ring_slot >> (8 * g)) & 0xFFu;
+            const uint32_t sl = (uint32_t)g * NSG + gs;
+            if (!(ok = mbar_wait(&empty[sl], ((ring_phase >> g) & 1u) ^ 1u, a.err, 2))) break;
+            unsigned char *dst = slots + (size_t)sl * L.slot_bytes;
             const uint32_t bytes = (uint32_t)(rows * T * ES + (m0 == 0 ? T * 4 : 0));
-            mbar_expect_tx(&full[slot], bytes);
-            if (m0 == 0) bulk_load(dst, s.V + (int64_t)i * ldx + col0, T * 4, &full[slot]);
-            const unsigned char *src = G + ((int64_t)i * s.ld_k + (int64_t)m0 * s.ld_m + col0) * ES;
-            for (int r = 0; r < rows; ++r)
-              bulk_load(dst + T * 4 + (size_t)r * T * ES, src + (int64_t)r * s.ld_m * ES, T * ES, &full[slot]);
-            if (++slot == (uint32_t)NS) { slot = 0; phase ^= 1; }
+            mbar_expect_tx(&full[sl], bytes);
+            if (m0 == 0) tma_load_2d(dst, &a.vmap, c0, i, &full[sl]);
+            if (rows > 0) tma_load_3d(dst + T * 4, &a.gmap[rows - 1], c0, m0, i, &full[sl]);
+            if (gs + 1 == (uint32_t)NSG) {
+              ring_slot &= ~(0xFFu << (8 * g));
+              ring_phase ^= 1u << g;
+            } else {
+              ring_slot += 1u << (8 * g);
+            }
             m0 += R;
           } while (m0 < n);
         }
       }
     }
   } else {
-    // ------------------------------------------------------------------ consumers (T/4 threads)
+    // ------------------------------------------------- consumers: NG groups of T/4 threads each
+    // Group g owns the learners i with i % NG == g (their updates are independent of each other
+    // once the old models are staged), so several ring items are consumed concurrently.
     const int ct = threadIdx.x - 32;
-    const int nq = T / 4;  // float4 per staged row
-    if (ct < nq) {
-      const float4 *xs4 = reinterpret_cast<const float4 *>(xs);
-      float4 *xs4w = reinterpret_cast<float4 *>(xs);
+    const int nq = T / 4;  // float4 per staged row = threads per group
+    const int grp = ct / nq, cq = ct - grp * nq;
+    {
       const float lr = s.lr, mom = s.mom;
+      const bool mix_first = s.order == NB_ORDER_MIX_THEN_UPDATE;
       uint32_t slot = 0, phase = 0;
       int titer = 0;
       for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x, ++titer) {
-        const int64_t col0 = (int64_t)tile * T + (int64_t)ct * 4;
+        const int64_t col0 = (int64_t)tile * T + (int64_t)cq * 4;
         float *Xc = s.X + col0;
         float *Vc = s.V + col0;
-        ok = __all_sync(0xffffffffu, mbar_wait(xfull, titer & 1, a.err, 3));  // warp-uniform outcome
+        const int xb = titer & 1;
+        float4 *xs4w = reinterpret_cast<float4 *>(xs_base + (size_t)xb * K * T);
+        const float4 *xs4 = xs4w;
+        ok = __all_sync(0xffffffffu, mbar_wait(&xfull[xb], (titer >> 1) & 1, a.err, 3));  // warp-uniform outcome
         if (!ok) break;
-        const bool mix_first = s.order == NB_ORDER_MIX_THEN_UPDATE;
         float4 mean = make_float4(0.f, 0.f, 0.f, 0.f);
         if (MEAN && mix_first) {
-          for (int j = 0; j < K; ++j) mean = add4(mean, xs4[j * nq + ct]);
+          for (int j = 0; j < K; ++j) mean = add4(mean, xs4[j * nq + cq]);
           mean = scale4(mean, s.inv_K);
         }
-        for (int i = 0; ok && i < K; ++i) {
+        for (int i = grp; ok && i < K; i += NG) {  // this group's learners, from its own ring
           const int n = s.n[i];
           float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
           float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
           int m0 = 0;
           do {
             const int rows = (n - m0 < R) ? (n - m0) : R;
-            ok = __all_sync(0xffffffffu, mbar_wait(&full[slot], phase, a.err, 4));
+            const uint32_t sl = (uint32_t)grp * NSG + slot;
+            ok = __all_sync(0xffffffffu, mbar_wait(&full[sl], phase, a.err, 4));
             if (!ok) break;
-            const unsigned char *src = slots + (size_t)slot * L.slot_bytes;
-            if (m0 == 0) v = reinterpret_cast<const float4 *>(src)[ct];
-            const unsigned char *rowp = src + T * 4 + (size_t)ct * 4 * ES;
+            const unsigned char *src = slots + (size_t)sl * L.slot_bytes;
+            if (m0 == 0) v = reinterpret_cast<const float4 *>(src)[cq];
+            const unsigned char *rowp = src + T * 4 + (size_t)cq * 4 * ES;
             for (int r = 0; r < rows; ++r) {
               Raw<SRC> raw;
               if constexpr (ES == 2) raw.r = *reinterpret_cast<const uint2 *>(rowp + (size_t)r * T * ES);
@@ -227,8 +286,8 @@ __global__ void __launch_bounds__(32 + 256, 2) nb_step_pipeline_kernel(const __g
               acc = add4(acc, widen(raw));
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&empty[slot]);
-            if (++slot == (uint32_t)NS) { slot = 0; phase ^= 1; }
+            if (lane == 0) mbar_arrive(&empty[sl]);
+            if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
             m0 += R;
           } while (m0 < n);
           if (!ok) break;
@@ -237,28 +296,34 @@ __global__ void __launch_bounds__(32 + 256, 2) nb_step_pipeline_kernel(const __g
           if (mix_first) {
             float4 xh;
             if constexpr (MEAN) xh = mean;
-            else xh = mix_row(xs4, nq, ct, s_col, s_val, s_beg[i], s_end[i]);
+            else xh = mix_row(xs4, nq, cq, s_col, s_val, s_beg[i], s_end[i]);
             st4(Xc + (int64_t)i * ldx, descend(xh, lr, vn));
           } else {
-            const float4 y = descend(xs4[i * nq + ct], lr, vn);
-            if constexpr (MEAN) mean = add4(mean, y);
-            else xs4w[i * nq + ct] = y;
+            xs4w[i * nq + cq] = descend(xs4[i * nq + cq], lr, vn);  // y_i replaces x_i in the stage
           }
         }
         if (!ok) break;
         if (!mix_first) {
+          // every group's y must be staged before anyone averages: bounded mbarrier rendezvous
+          __syncwarp();
+          if (lane == 0) mbar_arrive(ybar);
+          ok = __all_sync(0xffffffffu, mbar_wait(ybar, titer & 1, a.err, 5));
+          if (!ok) break;
           if constexpr (MEAN) {
-            const float4 m = scale4(mean, s.inv_K);
-            for (int i = 0; i < K; ++i) st4(Xc + (int64_t)i * ldx, m);
-          } else {
-            for (int i = 0; i < K; ++i)
-              st4(Xc + (int64_t)i * ldx, mix_row(xs4, nq, ct, s_col, s_val, s_beg[i], s_end[i]));
-            // the stage was written by this thread; order those writes before the next bulk copy
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            for (int j = 0; j < K; ++j) mean = add4(mean, xs4[j * nq + cq]);
+            mean = scale4(mean, s.inv_K);
           }
+          for (int i = grp; i < K; i += NG) {
+            float4 xn;
+            if constexpr (MEAN) xn = mean;
+            else xn = mix_row(xs4, nq, cq, s_col, s_val, s_beg[i], s_end[i]);
+            st4(Xc + (int64_t)i * ldx, xn);
+          }
+          // the stage was written through the generic proxy; order that before the next bulk copy
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(xempty);
+        if (lane == 0) mbar_arrive(&xempty[xb]);
       }
     }
   }
@@ -266,7 +331,7 @@ __global__ void __launch_bounds__(32 + 256, 2) nb_step_pipeline_kernel(const __g
 }
 
 struct PipeTuning {
-  int enabled = 1, T = 0, slots = 0, ctas_per_sm = 0, rows = 0;
+  int enabled = 1, T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0;
   int sm_count = 0;
 };
 
@@ -282,12 +347,51 @@ PipeTuning &tuning() {
     q.slots = geti("NB_PIPELINE_SLOTS", 0);
     q.ctas_per_sm = geti("NB_PIPELINE_CTAS_PER_SM", 0);
     q.rows = geti("NB_PIPELINE_ROWS", 0);
+    q.groups = geti("NB_PIPELINE_GROUPS", 0);
     return q;
   }();
   return t;
 }
 
 constexpr int kSmemBudget = 227 * 1024;
+
+using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                              const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (no link against libcuda).
+EncodeFn encode_fn() {
+  static EncodeFn fn = [] {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    cudaGetLastError();
+    return reinterpret_cast<EncodeFn>(p);
+  }();
+  return fn;
+}
+
+CUtensorMapDataType unit_type(int bytes) {
+  switch (bytes) {
+    case 1: return CU_TENSOR_MAP_DATA_TYPE_UINT8;
+    case 2: return CU_TENSOR_MAP_DATA_TYPE_UINT16;
+    case 4: return CU_TENSOR_MAP_DATA_TYPE_UINT32;
+    default: return CU_TENSOR_MAP_DATA_TYPE_UINT64;
+  }
+}
+
+// Rows of `row_bytes`-pitched data seen as [outer..., units]: the innermost extent covers exactly the
+// full tiles, so no copy ever touches a ragged edge.
+bool encode_map(CUtensorMap *map, const void *base, int unit_bytes, int rank, const cuuint64_t *dims,
+                const cuuint64_t *strides, const cuuint32_t *box) {
+  const cuuint32_t ones[3] = {1, 1, 1};
+  return encode_fn()(map, unit_type(unit_bytes), (cuuint32_t)rank, const_cast<void *>(base), dims, strides, box, ones,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 
 }  // namespace
 
@@ -304,24 +408,40 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   }
   // bulk copies need 16-byte aligned sources and sizes
   if ((uintptr_t)a.G % 16 != 0 || (a.ld_m * es) % 16 != 0 || (a.ld_k * es) % 16 != 0) return false;
-  int T = t.T ? t.T : (a.K <= 16 ? 512 : (a.K <= 32 ? 256 : 128));
-  if (T % 128 != 0 || T < 128 || T > 1024) return false;
-  if (a.P < T) return false;
-  const int R = t.rows ? t.rows : (es == 2 ? 8 : 4);
-  const int ctas = t.ctas_per_sm ? t.ctas_per_sm : 2;
-  const int budget = kSmemBudget / ctas - 1024;
-  int slots = t.slots;
-  if (!slots) {
+  if (!encode_fn()) return false;
+  int R = t.rows ? t.rows : 8;
+  if (R < 1) R = 1;
+  if (R > kMaxRowsPerItem) R = kMaxRowsPerItem;
+  if (R > a.M) R = a.M;
+  // Tile width: a box row is 256 units of T*es/256 bytes, so T is 128, 256 or 512.  CTAs per SM and
+  // T shrink until the ring has at least 3 slots beside the double-buffered X stage.
+  int T = t.T ? t.T : 512;
+  int ctas = t.ctas_per_sm ? t.ctas_per_sm : 2;
+  int groups = 1, slots = 0;
+  for (;;) {
+    if (T != 128 && T != 256 && T != 512) return false;
+    groups = t.groups ? t.groups : 2;
+    if (groups > kMaxGroups) groups = kMaxGroups;
+    if (groups > a.K) groups = a.K;
+    while (groups > 1 && groups * (T / 4) > 512) --groups;
     const PipeLayout L0 = pipe_layout(a.K, T, es, R, 0, a.mix_slots);
-    slots = (budget - L0.total - 64) / (T * 4 + R * T * es);
-    if (slots > 24) slots = 24;
+    const int budget = kSmemBudget / ctas - 1024;
+    slots = (budget - L0.total - 256) / (T * 4 + R * T * es);
+    if (t.slots && t.slots < slots) slots = t.slots;
+    if (slots > 32) slots = 32;
+    slots -= slots % groups;  // every group's ring has the same number of slots
+    if (slots >= 2 * groups) break;
+    if (ctas > 1 && !t.ctas_per_sm) { --ctas; continue; }
+    if (T > 128 && !t.T) { T /= 2; continue; }
+    return false;
   }
-  if (slots < 2) return false;
+  if (a.P < T) return false;
   const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots);
   if (L.total > kSmemBudget) return false;
   plan->T = T;
   plan->rows_per_item = R;
   plan->n_slots = slots;
+  plan->n_groups = groups;
   plan->smem_bytes = L.total;
   plan->n_tiles = (int)(a.P / T);
   const int64_t max_ctas = (int64_t)ctas * t.sm_count;
@@ -342,13 +462,35 @@ cudaError_t configure_pipeline() {
 
 cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan, int *err_flag, cudaStream_t st) {
   PipeArgs p;
+  std::memset(&p, 0, sizeof(p));
   p.s = a;
   p.T = plan.T;
   p.n_slots = plan.n_slots;
   p.rows_per_item = plan.rows_per_item;
   p.n_tiles = plan.n_tiles;
+  p.n_groups = plan.n_groups;
   p.err = err_flag;
-  const int threads = 32 + plan.T / 4;
+  const cuuint64_t units = (cuuint64_t)plan.n_tiles * kBoxInner;
+  {  // X and V: [K, units] fp32 rows of pitch ldx
+    const int ub = plan.T * 4 / kBoxInner;
+    const cuuint64_t dims[2] = {units, (cuuint64_t)a.K};
+    const cuuint64_t strides[1] = {(cuuint64_t)a.ldx * 4};
+    const cuuint32_t xbox[2] = {kBoxInner, (cuuint32_t)a.K};
+    const cuuint32_t vbox[2] = {kBoxInner, 1};
+    if (!encode_map(&p.xmap, a.X, ub, 2, dims, strides, xbox) || !encode_map(&p.vmap, a.V, ub, 2, dims, strides, vbox))
+      return cudaErrorInvalidValue;
+  }
+  {  // G: [K, M, units]; one map per box height
+    const int ub = plan.T * es / kBoxInner;
+    const cuuint64_t dims[3] = {units, (cuuint64_t)a.M, (cuuint64_t)a.K};
+    const cuuint64_t strides[2] = {(cuuint64_t)a.ld_m * es, (cuuint64_t)a.ld_k * es};
+    const int rmax = plan.rows_per_item < a.M ? plan.rows_per_item : a.M;
+    for (int r = 1; r <= rmax; ++r) {
+      const cuuint32_t box[3] = {kBoxInner, (cuuint32_t)r, 1};
+      if (!encode_map(&p.gmap[r - 1], a.G, ub, 3, dims, strides, box)) return cudaErrorInvalidValue;
+    }
+  }
+  const int threads = 32 + plan.n_groups * (plan.T / 4);
   if (es == 2) {
     if (a.mean_mode) nb_step_pipeline_kernel<2, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
     else nb_step_pipeline_kernel<2, false><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
