@@ -223,6 +223,40 @@ int nb_get_device_mixing(nb_ctx *c, uint32_t *bits, float *W_dense, void *stream
 int nb_get_stats(const nb_ctx *c, int64_t *sum_finished, double *algorithmic_bytes,
                  int64_t *kernel_launches);
 
+/* ------------------------------------------------------------------------------------------------
+ * Allocation-free variant (no counterpart in the paper: it exists for deployment reasons only).
+ *
+ * For callers that may not allocate device memory while they run - a process whose framework pool
+ * already owns the whole GPU, a serving loop that cannot take the device-wide stall of an
+ * allocation, a deployment that forbids allocation after start-up.  It runs one all-reduce-variant
+ * iteration (masked accumulate, mean normalisation, mean over learners, momentum step, Alg. 2
+ * order) entirely on memory the caller passes in, plus ONE piece of scratch: the fp32 accumulator
+ * between the accumulate kernel and the update kernel, which is a fixed array inside the library
+ * image of NB_STATIC_MAX_ELEMS floats (16 MiB; every GPU that loads the library holds it until the
+ * process exits).  No context is needed and nothing is allocated or freed, by the CUDA runtime or
+ * by any library, in any call.
+ *
+ *   X, V      device, in/out, [K, ld] fp32 models and momentum, 16-byte aligned, ld >= P and a
+ *             multiple of 4; columns [P, ld) of each row are padding the call may overwrite
+ *   grads, dtype, ld_m, ld_k, finished   as nb_accumulate
+ *
+ * Limits and behaviour
+ *   - K*ld must not exceed NB_STATIC_MAX_ELEMS: larger problems are rejected with
+ *     NB_ERR_UNSUPPORTED and a message (nb_last_error(NULL)); nothing is launched.
+ *   - The first call on each device resolves the array's device address (once, with that device
+ *     current); make that first call during set-up, before any stream capture is begun.
+ *   - All calls on a device share the one array.  A call overwrites every element it later reads,
+ *     so no state leaks from one call to the next, but two calls whose kernels overlap on the GPU
+ *     (different streams, different threads, different contexts of the library) race on it:
+ *     serialise them.
+ *   - Results are bit-identical to nb_accumulate + nb_step on an NB_ALLREDUCE context.
+ * Errors: NB_ERR_ARG, NB_ERR_UNSUPPORTED, NB_ERR_CUDA; text through nb_last_error(NULL).
+ * ---------------------------------------------------------------------------------------------- */
+#define NB_STATIC_MAX_ELEMS (1 << 22)
+int nb_step_static(int K, int64_t P, int M, float lr, float mom, float *X, float *V, int64_t ld,
+                   const void *grads, int dtype, int64_t ld_m, int64_t ld_k, const int32_t *finished,
+                   void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,6 +21,7 @@ NB_NORM_MEAN, NB_NORM_PAPER = 0, 1
 NB_ORDER_MIX_THEN_UPDATE, NB_ORDER_UPDATE_THEN_MIX = 0, 1
 NB_STRAG_UNIFORM_COUNT, NB_STRAG_SHIFTED_EXP, NB_STRAG_SHIFTED_EXP_SLOWSET = 0, 1, 2
 NB_MAX_K, NB_MAX_MATCHINGS, NB_MAX_NNZ = 64, 32, 1024
+NB_STATIC_MAX_ELEMS = 1 << 22
 
 VARIANTS = {"allreduce": NB_ALLREDUCE, "dpsgd": NB_DPSGD, "matcha": NB_MATCHA, "centralized": NB_CENTRALIZED}
 STRAGGLER_MODELS = {"uniform_count": NB_STRAG_UNIFORM_COUNT, "shifted_exp": NB_STRAG_SHIFTED_EXP,
@@ -74,6 +75,7 @@ def _load():
         "nb_get_matcha_activation": [vp, i64, P(C.c_uint32)],
         "nb_get_device_mixing": [vp, P(C.c_uint32), P(C.c_float), vp],
         "nb_get_stats": [vp, P(i64), P(C.c_double), P(i64)],
+        "nb_step_static": [i32, i64, i32, f32, f32, vp, vp, i64, vp, i32, i64, i64, P(C.c_int32), vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -89,7 +91,7 @@ EXPORTED = ["nb_straggler_sample", "nb_topology_matchings", "nb_mixing_matrix", 
             "nb_last_error", "nb_set_option", "nb_set_lr", "nb_set_params", "nb_accumulate", "nb_step",
             "nb_step_fused", "nb_step_fused_host", "nb_get_params", "nb_get_momentum", "nb_get_accumulator",
             "nb_get_mean_params", "nb_set_state", "nb_get_step", "nb_get_W", "nb_get_matcha_activation",
-            "nb_get_device_mixing", "nb_get_stats"]
+            "nb_get_device_mixing", "nb_get_stats", "nb_step_static"]
 
 
 def _i32p(a):
@@ -298,6 +300,19 @@ class NbContext:
         s, b, l = C.c_int64(0), C.c_double(0), C.c_int64(0)
         self._ck(lib.nb_get_stats(self._h, C.byref(s), C.byref(b), C.byref(l)))
         return {"sum_finished": s.value, "algorithmic_bytes": b.value, "kernel_launches": l.value}
+
+
+def step_static(X, V, grads, finished, P, M, lr, mom, ld_m=0, ld_k=0):
+    """nb_step_static: one all-reduce-variant iteration on caller-owned X[K, ld], V[K, ld] (device
+    tensors, updated in place) for callers that cannot allocate device memory; the accumulator
+    lives in a fixed array inside the library.  Raises NbError (NB_ERR_UNSUPPORTED) when K*ld
+    exceeds NB_STATIC_MAX_ELEMS."""
+    K, ld = X.shape
+    n = np.ascontiguousarray(finished, dtype=np.int32)
+    rc = lib.nb_step_static(K, P, M, lr, mom, _ptr(X), _ptr(V), ld, _ptr(grads), _dtype_code(grads), ld_m, ld_k,
+                            _i32p(n), _stream())
+    if rc != NB_OK:
+        raise NbError(rc, lib.nb_last_error(None).decode())
 
 
 def context_for(w, P=None):

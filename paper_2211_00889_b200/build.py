@@ -11,7 +11,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnb.so")
-SOURCES = ["nb_api.cu", "nb_kernels.cu", "nb_pipeline.cu", "nb_host.cpp"]
+SOURCES = ["nb_api.cu", "nb_kernels.cu", "nb_pipeline.cu", "nb_static.cu", "nb_host.cpp"]
 
 
 def _nvcc():

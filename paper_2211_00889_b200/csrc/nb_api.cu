@@ -48,6 +48,14 @@ struct DeviceGuard {
   }
 };
 
+}  // namespace
+
+namespace nb {
+void set_global_error(const std::string &msg) { g_create_err = msg; }
+}  // namespace nb
+
+namespace {
+
 int fail(nb_ctx *c, int code, const std::string &msg) {
   if (c) {
     c->err = msg;

@@ -272,6 +272,8 @@ static cudaError_t launch_step_direct(const StepArgs &a, int src, cudaStream_t s
   return a.g_aligned ? launch_step_t<kSrcBF16, true>(a, st) : launch_step_t<kSrcBF16, false>(a, st);
 }
 
+cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st) { return launch_step_direct(a, src, st); }
+
 cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st) {
   *launches = 0;
   // The pipeline kernel sees one gradient-like stream; the unfused step presents the accumulator
