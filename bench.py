@@ -33,10 +33,11 @@ METRIC = "fused NB-SGD step throughput (params*learners/s)"
 UNIT = "params*learners/s"
 DEFAULT_WORKLOAD = "cfg3_dpsgd_ring_resnet50"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per algorithmic byte of the fused step kernel, from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of the
-# captured launch); None until a capture exists.
-TRAFFIC_PER_ALGORITHMIC_BYTE = None
+# DRAM bytes per algorithmic byte of the fused step kernel: dram__bytes_read.sum + dram__bytes_write.sum
+# of nb_step_pipeline_kernel over the algorithmic bytes of the same launch, from the ncu capture of an
+# 8M-column case of the default workload (profiles/nb_step_pipeline_kernel_cfg3_8Mcols_traffic.md).
+# Traffic grows in proportion to the columns a launch processes.
+TRAFFIC_PER_ALGORITHMIC_BYTE = 0.988
 
 
 def parse_args():
@@ -192,9 +193,10 @@ def run_ours(args, w):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
+    from paper_2211_00889_b200 import sharding
+
     def barrier():
-        if world > 1:
-            dist.barrier()
+        sharding.barrier()
         torch.cuda.synchronize()
 
     # rank r owns columns [r*P, (r+1)*P) of an N*P-wide problem: same counts everywhere, own data
@@ -218,6 +220,8 @@ def run_ours(args, w):
     total_steps = args.warmup + args.steps
     for t in range(args.warmup):
         ctx.step_fused(bufs[t % n_buf], counts(t))
+    if world > 1:   # every rank derives the counts by itself; they must coincide (checked outside the timed region)
+        assert sharding.counts_agree(counts(args.warmup), dev), "ranks disagree on the finished counts"
     barrier()
     launches0 = ctx.get_stats()["kernel_launches"]
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
@@ -242,10 +246,7 @@ def run_ours(args, w):
     launches = ctx.get_stats()["kernel_launches"] - launches0
     total_ms = e0.elapsed_time(e1)
     launch_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
-    tmax = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    total_ms_max = float(tmax.item())
+    total_ms_max = sharding.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms_max / args.steps
     value = w.K * w.P * world / (ms_per_step * 1e-3)
 
@@ -254,7 +255,7 @@ def run_ours(args, w):
     achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_per_launch) if TRAFFIC_PER_ALGORITHMIC_BYTE else None,
-                "peak_source": "of " + peak_kind, "kernel": "nb_step_kernel (fused accumulate+mix+momentum+update)",
+                "peak_source": "of " + peak_kind, "kernel": "nb_step_pipeline_kernel (fused accumulate+mix+momentum+update)",
                 "algorithmic_bytes_per_launch": bytes_per_launch, "launch_ms": launch_ms,
                 "frac_of_8TBps_nominal": achieved / 8000.0, "mean_sum_finished": sum_n / args.steps}
 
@@ -279,10 +280,7 @@ def run_ours(args, w):
         barrier()
         wall = time.perf_counter() - t0
         dev_ms = a0.elapsed_time(a1)
-        tm = torch.tensor([max(dev_ms, wall * 1e3)], device=dev, dtype=torch.float64)
-        if world > 1:
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        per = float(tm.item()) / args.e2e_steps
+        per = sharding.max_over_ranks(max(dev_ms, wall * 1e3), dev) / args.e2e_steps
         e2e = {"value": w.K * w.P * world / (per * 1e-3), "unit": UNIT, "ms_per_step": per,
                "steps": args.e2e_steps, "h2d_bytes_per_step": h2d // args.e2e_steps,
                "d2h_bytes_per_step": w.P * 4,
