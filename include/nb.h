@@ -125,6 +125,25 @@ typedef struct nb_straggler {
 int nb_straggler_sample(const nb_straggler *cfg, int K, int M, int64_t step, int32_t *finished,
                         uint8_t *mask, double *tau);
 
+/* Run-time figures of the straggler model over `steps` iterations starting at step0 (Sec. 4.2-4.3):
+ * per-iteration run-time of Non-blocking SGD, M*min_i tau_i (Lemma 1: the first order statistic),
+ * and of a blocking method, M*max_i tau_i; their ratio (Theorem 1); the throughput ratio
+ * Y*X_{K:K}/K with Y = sum_i 1/tau_i (Theorem 5); the data fraction Y*X_{1:K}/K that Corollary 1
+ * predicts for fractional mini-batches, and the fraction sum_i n_i/(K*M) the floor rule yields.
+ * Host only.  NB_ERR_UNSUPPORTED for NB_STRAG_UNIFORM_COUNT (it has no times). */
+typedef struct nb_runtime_report {
+  double mean_t_nonblocking;    /* mean of M * min_i tau_i                     */
+  double mean_t_blocking;       /* mean of M * max_i tau_i                     */
+  double ratio;                 /* mean_t_nonblocking / mean_t_blocking        */
+  double mean_throughput_ratio; /* mean of Y * max_i tau_i / K                 */
+  double mean_fractional_data;  /* mean of Y * min_i tau_i / K                 */
+  double mean_finished_fraction;/* mean of sum_i n_i / (K*M)                   */
+  double mean_min_tau, mean_max_tau;
+  int64_t steps;
+} nb_runtime_report;
+int nb_runtime_report_compute(const nb_straggler *cfg, int K, int M, int64_t step0, int64_t steps,
+                              nb_runtime_report *out);
+
 /* ------------------------------------------------------------------------------------------------
  * Host topology helpers (no context, no GPU).
  * ---------------------------------------------------------------------------------------------- */
@@ -178,6 +197,19 @@ int nb_set_params(nb_ctx *c, const float *x0, int per_learner, void *stream);
  * finished: host [K], each in [0, M].  Errors: NB_ERR_ARG. */
 int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
                   const int32_t *finished, void *stream);
+
+/* Streaming form of step 1 (Alg. 1 inner loop as the gradients arrive): a learner hands over one
+ * finished mini-batch gradient at a time.  nb_begin_iteration clears the per-learner counts and the
+ * terminal signal.  nb_accumulate_minibatch adds grad[P] (device, NB_F32 or NB_BF16) to learner i's
+ * accumulator in fp32 - the same sums, in the same order, as nb_accumulate - and counts it; when a
+ * learner has delivered all M mini-batches it is the first finisher and the terminal signal is
+ * raised ("Broadcast terminal signals if n = N"); every later call of the iteration returns
+ * NB_ABANDONED (a status, not an error) without touching anything ("Break and abandon unfinished
+ * mini-batches").  nb_step then runs on the counts collected.  nb_get_finished reports them. */
+#define NB_ABANDONED 1
+int nb_begin_iteration(nb_ctx *c);
+int nb_accumulate_minibatch(nb_ctx *c, int learner, const void *grad, int dtype, void *stream);
+int nb_get_finished(const nb_ctx *c, int32_t *finished /* host out [K] */, int32_t *terminal /* host out or NULL */);
 
 /* Steps 2-4 on what the last nb_accumulate stored; advances the step counter.
  * NB_ERR_STATE if there has been no nb_accumulate since the last step. */

@@ -143,6 +143,40 @@ def straggler_counts(model, seed, t, K, M, params=()):
     raise ValueError(model)
 
 
+def runtime_report(model, seed, K, M, steps, params=(), step0=0):
+    """Run-time figures of the straggler model averaged over `steps` iterations (Sec. 4.2-4.3):
+    Non-blocking SGD waits for the fastest learner, M*min(tau) per iteration (Lemma 1); a blocking
+    method waits for the slowest, M*max(tau); their ratio is Theorem 1's; the throughput ratio is
+    Theorem 5's Y*X_{K:K}/K with Y = sum_i 1/tau_i; Corollary 1's data per iteration, as a fraction
+    of K batches, is Y*X_{1:K}/K; the floor rule gives sum n_i/(K*M)."""
+    t_nb = t_bl = thr = frac = fin = tmin_s = tmax_s = 0.0
+    for t in range(step0, step0 + steps):
+        if model == "shifted_exp":
+            delta = [params[0]] * K
+        elif model == "shifted_exp_slowset":
+            slow = set(slow_set(seed, t, K, int(math.floor(params[0] * K))))
+            delta = [params[1] if i in slow else params[2] for i in range(K)]
+        else:
+            raise ValueError(model)
+        tau = delays_shifted_exp(seed, t, K, delta)
+        n = counts_from_delays(tau, M)
+        Y = 0.0
+        for x in tau:
+            Y += 1.0 / x
+        t_nb += float(M) * min(tau)
+        t_bl += float(M) * max(tau)
+        thr += Y * max(tau) / float(K)
+        frac += Y * min(tau) / float(K)
+        fin += float(sum(n)) / (float(K) * float(M))
+        tmin_s += min(tau)
+        tmax_s += max(tau)
+    inv = 1.0 / float(steps)
+    return {"mean_t_nonblocking": t_nb * inv, "mean_t_blocking": t_bl * inv, "ratio": t_nb / t_bl,
+            "mean_throughput_ratio": thr * inv, "mean_fractional_data": frac * inv,
+            "mean_finished_fraction": fin * inv, "mean_min_tau": tmin_s * inv, "mean_max_tau": tmax_s * inv,
+            "steps": steps}
+
+
 def finished_mask(n, M):
     """mask[i][m] = 1 iff mini-batch m of learner i was finished; unfinished ones are a suffix
     because a learner leaves its loop at the terminal signal (Alg. 1 inner loop)."""

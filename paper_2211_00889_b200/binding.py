@@ -22,6 +22,7 @@ NB_ORDER_MIX_THEN_UPDATE, NB_ORDER_UPDATE_THEN_MIX = 0, 1
 NB_STRAG_UNIFORM_COUNT, NB_STRAG_SHIFTED_EXP, NB_STRAG_SHIFTED_EXP_SLOWSET = 0, 1, 2
 NB_MAX_K, NB_MAX_MATCHINGS, NB_MAX_NNZ = 64, 32, 1024
 NB_STATIC_MAX_ELEMS = 1 << 22
+NB_ABANDONED = 1
 
 VARIANTS = {"allreduce": NB_ALLREDUCE, "dpsgd": NB_DPSGD, "matcha": NB_MATCHA, "centralized": NB_CENTRALIZED}
 STRAGGLER_MODELS = {"uniform_count": NB_STRAG_UNIFORM_COUNT, "shifted_exp": NB_STRAG_SHIFTED_EXP,
@@ -33,6 +34,13 @@ class nb_topology(C.Structure):
                 ("row_ptr", C.POINTER(C.c_int32)), ("col_idx", C.POINTER(C.c_int32)), ("val", C.POINTER(C.c_float)),
                 ("n_matchings", C.c_int32), ("partner", C.POINTER(C.c_int32)),
                 ("alpha", C.c_float), ("act_prob", C.c_float)]
+
+
+class nb_runtime_report(C.Structure):
+    _fields_ = [("mean_t_nonblocking", C.c_double), ("mean_t_blocking", C.c_double), ("ratio", C.c_double),
+                ("mean_throughput_ratio", C.c_double), ("mean_fractional_data", C.c_double),
+                ("mean_finished_fraction", C.c_double), ("mean_min_tau", C.c_double), ("mean_max_tau", C.c_double),
+                ("steps", C.c_int64)]
 
 
 class nb_straggler(C.Structure):
@@ -75,6 +83,10 @@ def _load():
         "nb_get_matcha_activation": [vp, i64, P(C.c_uint32)],
         "nb_get_device_mixing": [vp, P(C.c_uint32), P(C.c_float), vp],
         "nb_get_stats": [vp, P(i64), P(C.c_double), P(i64)],
+        "nb_begin_iteration": [vp],
+        "nb_accumulate_minibatch": [vp, i32, vp, i32, vp],
+        "nb_get_finished": [vp, P(C.c_int32), P(C.c_int32)],
+        "nb_runtime_report_compute": [P(nb_straggler), i32, i32, i64, i64, P(nb_runtime_report)],
         "nb_step_static": [i32, i64, i32, f32, f32, vp, vp, i64, vp, i32, i64, i64, P(C.c_int32), vp],
     }
     for name, args in sig.items():
@@ -91,7 +103,8 @@ EXPORTED = ["nb_straggler_sample", "nb_topology_matchings", "nb_mixing_matrix", 
             "nb_last_error", "nb_set_option", "nb_set_lr", "nb_set_params", "nb_accumulate", "nb_step",
             "nb_step_fused", "nb_step_fused_host", "nb_get_params", "nb_get_momentum", "nb_get_accumulator",
             "nb_get_mean_params", "nb_set_state", "nb_get_step", "nb_get_W", "nb_get_matcha_activation",
-            "nb_get_device_mixing", "nb_get_stats", "nb_step_static"]
+            "nb_get_device_mixing", "nb_get_stats", "nb_step_static",
+            "nb_begin_iteration", "nb_accumulate_minibatch", "nb_get_finished", "nb_runtime_report_compute"]
 
 
 def _i32p(a):
@@ -139,6 +152,20 @@ def straggler_sample(model, seed, step, K, M, params=()):
     if rc != NB_OK:
         raise NbError(rc, "nb_straggler_sample")
     return n, mask, tau
+
+
+def runtime_report(model, seed, K, M, steps, params=(), step0=0):
+    """nb_runtime_report_compute as a dict (host only)."""
+    cfg = nb_straggler()
+    cfg.model = STRAGGLER_MODELS[model] if isinstance(model, str) else model
+    cfg.seed = seed
+    for q, v in enumerate(params):
+        cfg.params[q] = float(v)
+    rep = nb_runtime_report()
+    rc = lib.nb_runtime_report_compute(C.byref(cfg), K, M, step0, steps, C.byref(rep))
+    if rc != NB_OK:
+        raise NbError(rc, "nb_runtime_report_compute")
+    return {name: getattr(rep, name) for name, _ in nb_runtime_report._fields_}
 
 
 def topology_matchings(topo, K):
@@ -234,6 +261,23 @@ class NbContext:
     def accumulate(self, grads, finished, ld_m=0, ld_k=0):
         n = self._finished(finished)
         self._ck(lib.nb_accumulate(self._h, _ptr(grads), _dtype_code(grads), ld_m, ld_k, _i32p(n), _stream()))
+
+    def begin_iteration(self):
+        self._ck(lib.nb_begin_iteration(self._h))
+
+    def accumulate_minibatch(self, learner, grad):
+        """True if the mini-batch was accumulated, False if it was abandoned (terminal signal raised)."""
+        rc = lib.nb_accumulate_minibatch(self._h, learner, _ptr(grad), _dtype_code(grad), _stream())
+        if rc == NB_ABANDONED:
+            return False
+        self._ck(rc)
+        return True
+
+    def get_finished(self):
+        n = np.zeros(self.K, dtype=np.int32)
+        term = C.c_int32(0)
+        self._ck(lib.nb_get_finished(self._h, _i32p(n), C.byref(term)))
+        return n, bool(term.value)
 
     def step(self):
         self._ck(lib.nb_step(self._h, _stream()))

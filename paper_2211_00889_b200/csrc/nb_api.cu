@@ -26,6 +26,7 @@ struct nb_ctx {
   int64_t step = 0;
   bool acc_fresh = false, device_mix_valid = false;
   int32_t n_acc[NB_MAX_K] = {0};
+  bool streaming = false, terminal = false;  // nb_begin_iteration / nb_accumulate_minibatch state
   int acc_esize = 4;
   int64_t sum_finished = 0, launches = 0;
   double alg_bytes = 0.0;
@@ -358,12 +359,53 @@ int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t
   std::memcpy(c->n_acc, a.n, sizeof(c->n_acc));
   c->acc_esize = es;
   c->acc_fresh = true;
+  c->streaming = false;
+  return NB_OK;
+}
+
+int nb_begin_iteration(nb_ctx *c) {
+  NB_ENTER(c);
+  std::memset(c->n_acc, 0, sizeof(c->n_acc));
+  c->streaming = true;
+  c->terminal = false;
+  c->acc_fresh = true;
+  c->acc_esize = 4;
+  return NB_OK;
+}
+
+int nb_accumulate_minibatch(nb_ctx *c, int learner, const void *grad, int dtype, void *stream) {
+  NB_ENTER(c);
+  if (!c->streaming) return fail(c, NB_ERR_STATE, "nb_accumulate_minibatch needs nb_begin_iteration first");
+  if (learner < 0 || learner >= c->K) return fail(c, NB_ERR_ARG, "learner index out of range");
+  if (!grad) return fail(c, NB_ERR_ARG, "grad is NULL");
+  if (dtype != NB_F32 && dtype != NB_BF16) return fail(c, NB_ERR_ARG, "dtype must be NB_F32 or NB_BF16");
+  if (c->terminal) return NB_ABANDONED;  // the first finisher has ended the iteration
+  const int es = dtype == NB_F32 ? 4 : 2;
+  const bool aligned = (uintptr_t)grad % (size_t)(4 * es) == 0;
+  NB_CUDA(c, nb::launch_add_minibatch(c->acc + (int64_t)learner * c->ldx, grad, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16,
+                                      aligned, c->P, c->n_acc[learner] == 0, (cudaStream_t)stream));
+  c->launches++;
+  c->acc_esize = es;
+  if (++c->n_acc[learner] == c->M) c->terminal = true;
+  return NB_OK;
+}
+
+int nb_get_finished(const nb_ctx *c, int32_t *finished, int32_t *terminal) {
+  if (!c || !finished) return NB_ERR_ARG;
+  for (int i = 0; i < c->K; ++i) finished[i] = c->n_acc[i];
+  if (terminal) *terminal = c->terminal ? 1 : 0;
   return NB_OK;
 }
 
 int nb_step(nb_ctx *c, void *stream) {
   NB_ENTER(c);
   if (!c->acc_fresh) return fail(c, NB_ERR_STATE, "nb_step needs an nb_accumulate since the last step");
+  if (c->streaming) {  // learners that delivered nothing contribute a zero accumulator
+    for (int i = 0; i < c->K; ++i)
+      if (c->n_acc[i] == 0)
+        NB_CUDA(c, cudaMemsetAsync(c->acc + (int64_t)i * c->ldx, 0, sizeof(float) * (size_t)c->ldx, (cudaStream_t)stream));
+    c->streaming = false;
+  }
   nb::StepArgs a;
   std::memset(&a, 0, sizeof(a));
   a.X = c->X;

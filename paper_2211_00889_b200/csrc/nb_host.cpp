@@ -318,3 +318,42 @@ extern "C" int nb_mixing_matrix(const nb_topology *topo, int variant, int K, int
   nb::dense_W(mx, step, W_dense, bits);
   return NB_OK;
 }
+
+extern "C" int nb_runtime_report_compute(const nb_straggler *cfg, int K, int M, int64_t step0, int64_t steps,
+                                         nb_runtime_report *out) {
+  if (!cfg || !out || K < 1 || K > NB_MAX_K || M < 1 || step0 < 0 || steps < 1) return NB_ERR_ARG;
+  if (cfg->model == NB_STRAG_UNIFORM_COUNT) return NB_ERR_UNSUPPORTED;
+  double tau[NB_MAX_K];
+  int32_t n[NB_MAX_K];
+  double s_nb = 0, s_bl = 0, s_thr = 0, s_frac = 0, s_fin = 0, s_min = 0, s_max = 0;
+  for (int64_t t = step0; t < step0 + steps; ++t) {
+    int rc = nb_straggler_sample(cfg, K, M, t, n, nullptr, tau);
+    if (rc != NB_OK) return rc;
+    double tmin = tau[0], tmax = tau[0], Y = 0.0;
+    int64_t fin = 0;
+    for (int i = 0; i < K; ++i) {
+      if (tau[i] < tmin) tmin = tau[i];
+      if (tau[i] > tmax) tmax = tau[i];
+      Y += 1.0 / tau[i];
+      fin += n[i];
+    }
+    s_min += tmin;
+    s_max += tmax;
+    s_nb += (double)M * tmin;
+    s_bl += (double)M * tmax;
+    s_thr += Y * tmax / (double)K;
+    s_frac += Y * tmin / (double)K;
+    s_fin += (double)fin / ((double)K * (double)M);
+  }
+  const double inv = 1.0 / (double)steps;
+  out->mean_t_nonblocking = s_nb * inv;
+  out->mean_t_blocking = s_bl * inv;
+  out->ratio = s_nb / s_bl;
+  out->mean_throughput_ratio = s_thr * inv;
+  out->mean_fractional_data = s_frac * inv;
+  out->mean_finished_fraction = s_fin * inv;
+  out->mean_min_tau = s_min * inv;
+  out->mean_max_tau = s_max * inv;
+  out->steps = steps;
+  return NB_OK;
+}

@@ -68,6 +68,19 @@ __global__ void __launch_bounds__(256) nb_accumulate_kernel(const __grid_constan
   st4(a.acc + (int64_t)i * a.ldx + col0, g);
 }
 
+// Streaming accumulate: acc_row = (first ? +0 : acc_row) + g, one mini-batch gradient at a time
+// (the same sum, in the same order, as nb_accumulate_kernel builds in one go).
+template <int SRC, bool ALIGNED>
+__global__ void __launch_bounds__(256) nb_add_minibatch_kernel(float *acc_row, const void *g, int64_t P, int first) {
+  const int64_t col0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * kColsPerThread;
+  if (col0 >= P) return;
+  const int nvalid = (P - col0 < 4) ? (int)(P - col0) : 4;
+  using E = typename ElemOf<SRC>::type;
+  const float4 r = widen(load_raw<ALIGNED>(reinterpret_cast<const E *>(g) + col0, nvalid, (Raw<SRC> *)nullptr));
+  float4 a = first ? make_float4(0.f, 0.f, 0.f, 0.f) : ld4(acc_row + col0);
+  st4(acc_row + col0, add4(a, r));
+}
+
 // -------------------------------------------------------------------------------------------------
 // K2 / K2f: normalise + momentum + mix + update (SRC = kSrcAcc), or the same fused with the masked
 // accumulate (SRC = kSrcF32 / kSrcBF16).
@@ -307,6 +320,19 @@ cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches
     ++*launches;
   }
   return cudaSuccess;
+}
+
+cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,
+                                 cudaStream_t st) {
+  const unsigned grid = (unsigned)((P + 1023) / 1024);
+  if (src == kSrcF32) {
+    if (aligned) nb_add_minibatch_kernel<kSrcF32, true><<<grid, 256, 0, st>>>(acc_row, g, P, first);
+    else nb_add_minibatch_kernel<kSrcF32, false><<<grid, 256, 0, st>>>(acc_row, g, P, first);
+  } else {
+    if (aligned) nb_add_minibatch_kernel<kSrcBF16, true><<<grid, 256, 0, st>>>(acc_row, g, P, first);
+    else nb_add_minibatch_kernel<kSrcBF16, false><<<grid, 256, 0, st>>>(acc_row, g, P, first);
+  }
+  return cudaGetLastError();
 }
 
 cudaError_t launch_centralized(const StepArgs &a, int src, cudaStream_t st) {

@@ -64,6 +64,8 @@ cudaError_t launch_accumulate(const StepArgs &a, int src, cudaStream_t st);
 cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st);
 // The direct-load step kernel on all P columns (no pipeline kernel, no device error word).
 cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st);
+cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,
+                                 cudaStream_t st);
 cudaError_t launch_centralized(const StepArgs &a, int src, cudaStream_t st);
 cudaError_t launch_matcha_build(const MatchaArgs &a, cudaStream_t st);
 cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, cudaStream_t st);

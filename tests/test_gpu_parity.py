@@ -378,3 +378,42 @@ def test_error_reporting(B):
     assert st["sum_finished"] == 4 and st["kernel_launches"] == 2
     assert st["algorithmic_bytes"] == 100 * (4 * 4 + 16 * 4)
     ctx.close()
+
+
+def test_streaming_accumulate_follows_alg1_and_equals_batch_accumulate(B):
+    """Mini-batch gradients handed over one at a time (Alg. 1 inner loop): the first learner to deliver
+    all M raises the terminal signal, later deliveries are abandoned; sums equal nb_accumulate's bits."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 2 * 512 + 20, steps=3)
+    a, b = B.context_for(w), B.context_for(w)
+    orc = H.oracle_for(w, w.P)
+    x0 = WL.init_params(w)
+    for c in (a, b):
+        c.set_params(torch.from_numpy(x0).cuda())
+    orc.set_params(x0)
+    with pytest.raises(B.NbError):
+        a.accumulate_minibatch(0, torch.zeros(w.P, device="cuda"))          # needs nb_begin_iteration
+    for t in range(w.steps):
+        payload, values = WL.gradients_np(w, t)
+        g = H.to_device(payload)
+        n = H.lib_counts(B, w, t)                                            # who finishes how many
+        if t == 2:
+            n = n.copy(); n[3] = 0                                           # a learner that delivers nothing
+        a.begin_iteration()
+        # deliver round-robin, mini-batch m of every learner that gets that far; the fastest (n_i = M) last
+        for m in range(w.M):
+            for i in np.argsort(-n, kind="stable")[::-1]:
+                if m < n[i]:
+                    assert a.accumulate_minibatch(int(i), g[i, m]) is True
+        got, terminal = a.get_finished()
+        assert got.tolist() == n.tolist() and terminal == bool((n == w.M).any())
+        if terminal:
+            assert a.accumulate_minibatch(0, g[0, 0]) is False               # abandoned after the signal
+            assert a.get_finished()[0].tolist() == n.tolist()
+        b.accumulate(g, n)
+        assert torch.equal(a.get_accumulator()[n > 0], b.get_accumulator()[n > 0])
+        a.step(); b.step()
+        orc.step(values, n.tolist())
+        assert torch.equal(a.get_params(), b.get_params())
+    H.assert_close(a.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+    a.close(); b.close()

@@ -1,0 +1,130 @@
+"""Edge cases of the bulk-copy pipeline kernel and of its hand-over to the direct-load kernel:
+sizes around one tile, many learners, more mini-batches than one ring item holds, learners with
+nothing finished, and bitwise agreement between the two kernels on the same values."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from oracle import nb_oracle as O
+from paper_2211_00889_b200 import workloads as WL
+from tests import _harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding
+    return binding
+
+
+def _against_oracle(B, w, steps, counts=None, fused=True):
+    import torch
+    ctx = B.context_for(w)
+    orc = H.oracle_for(w, w.P)
+    x0 = WL.init_params(w)
+    ctx.set_params(torch.from_numpy(x0).cuda())
+    orc.set_params(x0)
+    launches = []
+    for t in range(steps):
+        n = counts[t] if counts is not None else H.lib_counts(B, w, t)
+        payload, values = WL.gradients_np(w, t)
+        before = ctx.get_stats()["kernel_launches"]
+        if fused:
+            ctx.step_fused(H.to_device(payload), n)
+        else:
+            ctx.accumulate(H.to_device(payload), n)
+            ctx.step()
+        launches.append(ctx.get_stats()["kernel_launches"] - before)
+        orc.step(values, [int(v) for v in n])
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT, w.name)
+    H.assert_close(ctx.get_momentum().numpy(), orc.V, H.TOL_SAME_INPUT, w.name)
+    ctx.close()
+    return launches
+
+
+@pytest.mark.parametrize("P,expected_launches", [
+    (512, 1),            # exactly one tile: pipeline kernel only
+    (512 + 8, 2),        # one tile + an 8-column tail for the direct kernel
+    (3 * 512, 1),
+    (511, 1),            # below one tile (and unaligned): direct kernel only
+    (256, 1),
+    (2 * 512 + 1, 1),    # odd row length: rows are not 16-byte aligned -> direct kernel only
+])
+def test_sizes_around_one_tile(B, P, expected_launches):
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], P, steps=3)
+    launches = _against_oracle(B, w, w.steps)
+    assert launches == [expected_launches] * w.steps
+
+
+@pytest.mark.parametrize("K", [2, 3, 17, 33, 64])
+@pytest.mark.parametrize("variant", ["dpsgd", "allreduce"])
+def test_learner_counts(B, K, variant):
+    base = WL.WORKLOADS["cfg3_dpsgd_ring_resnet50" if variant == "dpsgd" else "cfg2_allreduce_resnet18"]
+    w = replace(WL.scaled(base, 2 * 512 + 24, steps=3), K=K)
+    _against_oracle(B, w, w.steps)
+    _against_oracle(B, w, w.steps, fused=False)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("M", [1, 9, 20])
+def test_more_minibatches_than_one_ring_item(B, dtype, M):
+    w = replace(WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 3 * 512 + 16, steps=3), M=M, grad_dtype=dtype, K=6)
+    _against_oracle(B, w, w.steps)
+    rng = np.random.default_rng(M)
+    counts = [rng.integers(0, M + 1, w.K) for _ in range(w.steps)]      # includes learners with nothing finished
+    counts[1][:] = 0
+    counts[2][:] = M
+    _against_oracle(B, w, w.steps, counts=counts)
+
+
+def test_matcha_and_options_on_pipeline_sizes(B):
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg4_matcha_vgg16"], 4 * 512, steps=4)
+    for norm, order in ((B.NB_NORM_PAPER, B.NB_ORDER_UPDATE_THEN_MIX), (B.NB_NORM_MEAN, B.NB_ORDER_UPDATE_THEN_MIX)):
+        ctx = B.context_for(w)
+        ctx.set_option(B.NB_OPT_NORM, norm)
+        ctx.set_option(B.NB_OPT_ORDER, order)
+        orc = H.oracle_for(w, w.P, "paper" if norm == B.NB_NORM_PAPER else "mean", "update_then_mix")
+        x0 = WL.init_params(w)
+        ctx.set_params(torch.from_numpy(x0).cuda()); orc.set_params(x0)
+        for t in range(w.steps):
+            n = H.lib_counts(B, w, t)
+            payload, values = WL.gradients_np(w, t)
+            ctx.step_fused(H.to_device(payload), n)
+            orc.step(values, n.tolist())
+        H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+        ctx.close()
+
+
+@pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16"])
+@pytest.mark.parametrize("order", [0, 1])
+def test_pipeline_and_direct_kernels_agree_bitwise(B, name, order):
+    """The same values reach the library once as a 16-byte aligned stream (pipeline kernel + tail)
+    and once shifted by one element (rows lose their alignment, so the direct-load kernel with
+    scalar loads runs everything): identical bits."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS[name], 5 * 512 + 36, steps=3)
+    a, b = B.context_for(w), B.context_for(w)
+    for c in (a, b):
+        c.set_option(B.NB_OPT_ORDER, order)
+        c.set_params(torch.from_numpy(WL.init_params(w)).cuda())
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        g = H.to_device(WL.gradients_np(w, t)[0])
+        flat = torch.empty(g.numel() + 1, dtype=g.dtype, device="cuda")
+        shifted = flat[1:].view_as(g)
+        shifted.copy_(g)
+        la = a.get_stats()["kernel_launches"]
+        a.step_fused(g, n)
+        lb = b.get_stats()["kernel_launches"]
+        b.step_fused(shifted, n)
+        extra = 1 if w.variant == "matcha" else 0
+        assert a.get_stats()["kernel_launches"] - la == 2 + extra      # pipeline + tail
+        assert b.get_stats()["kernel_launches"] - lb == 1 + extra      # direct only
+    assert torch.equal(a.get_params(), b.get_params())
+    assert torch.equal(a.get_momentum(), b.get_momentum())
+    a.close(); b.close()

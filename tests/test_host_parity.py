@@ -135,3 +135,16 @@ def test_expected_finished_fraction_of_the_bench_workload():
     tot = sum(int(B.straggler_sample(w.straggler_model, w.seed, t, w.K, w.M, w.straggler_params)[0].sum())
               for t in range(3000))
     assert 70.0 < tot / 3000 < 77.0
+
+
+@pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg5_scale_ring"])
+def test_runtime_report_matches_oracle(name):
+    w = WORKLOADS[name]
+    got = B.runtime_report(w.straggler_model, w.seed, w.K, w.M, 400, w.straggler_params, step0=3)
+    want = O.runtime_report(w.straggler_model, w.seed, w.K, w.M, 400, w.straggler_params, step0=3)
+    assert got["steps"] == want["steps"] == 400
+    for k in want:
+        assert got[k] == pytest.approx(want[k], rel=1e-13), k
+    with pytest.raises(B.NbError) as e:
+        B.runtime_report("uniform_count", 1, 4, 4, 10)
+    assert e.value.code == B.NB_ERR_UNSUPPORTED

@@ -157,6 +157,26 @@ def test_slow_set_is_a_uniform_subset_without_repeats():
     assert tot_slow / c_slow < tot_fast / c_fast - 1.0
 
 
+def test_runtime_report_matches_theorems_1_and_2():
+    # tau = 1 + Exp(mean delta): E[min] = 1 + delta/K, E[max] = 1 + delta*H_K (Theorem 2, shifted by 1)
+    K, M, delta, steps = 10, 8, 1.0, 20000
+    rep = O.runtime_report("shifted_exp", 4242, K, M, steps, (delta,))
+    tnb, tdp = _theorem2_table()[(K, 1.0)]
+    se_min = (delta / K) / math.sqrt(steps)
+    se_max = delta * math.sqrt(sum(1.0 / k ** 2 for k in range(1, K + 1)) / steps)
+    assert abs(rep["mean_min_tau"] - (1.0 + tnb)) < 4 * se_min
+    assert abs(rep["mean_max_tau"] - (1.0 + tdp)) < 4 * se_max
+    assert rep["mean_t_nonblocking"] == pytest.approx(M * rep["mean_min_tau"], rel=1e-12)     # Lemma 1
+    assert rep["mean_t_blocking"] == pytest.approx(M * rep["mean_max_tau"], rel=1e-12)
+    assert rep["ratio"] == pytest.approx(rep["mean_t_nonblocking"] / rep["mean_t_blocking"], rel=1e-12)  # Theorem 1
+    assert rep["ratio"] < 1.0 < rep["mean_throughput_ratio"]                                   # Theorem 5: > 1
+    # floor rule never exceeds Corollary 1's fractional data, and is within one mini-batch per learner of it
+    assert rep["mean_fractional_data"] - 1.0 / M <= rep["mean_finished_fraction"] <= rep["mean_fractional_data"] + 1e-12
+    # no delay spread: everything is 1
+    rep0 = O.runtime_report("shifted_exp", 1, 4, 8, 50, (0.0,))
+    assert rep0["ratio"] == 1.0 and rep0["mean_throughput_ratio"] == 1.0 and rep0["mean_finished_fraction"] == 1.0
+
+
 def test_finished_mask_is_a_prefix():
     m = O.finished_mask([0, 1, 3, 4], 4)
     assert m.dtype == np.uint8
