@@ -2,22 +2,28 @@
 //
 // The step is bound by HBM bandwidth, and what limits a plain load/store kernel is the number of
 // bytes it can keep in flight: every outstanding load pins registers of a resident thread.  Here
-// the loads are issued by ONE producer thread per CTA as tiled bulk asynchronous copies (TMA:
-// cp.async.bulk.tensor through tensor maps, global -> shared, completion counted on an mbarrier),
-// so the bytes in flight are bounded by shared memory, not by occupancy, and one instruction moves
-// a whole box of rows (the producer is issue-bound with one instruction per row):
+// the loads are tiled bulk asynchronous copies (TMA: cp.async.bulk.tensor through tensor maps,
+// global -> shared, completion counted in bytes on an mbarrier) issued by a handful of producer
+// threads, so the bytes in flight are bounded by shared memory, not by occupancy, and one
+// instruction moves a whole box of rows (with one instruction per row the producers are
+// issue-bound):
 //
 //   * the CTA owns column tiles of T columns (persistent, tile = blockIdx.x + k * gridDim.x);
-//   * per tile the producer first brings the K old model rows X[:, tile] into the X stage with one
-//     box copy (the mix needs every neighbour's OLD value while X is updated in place), then
-//     streams, learner by learner, "items" into a ring of slots: item = momentum row V[i, tile]
-//     (one box) + up to R finished gradient rows G[i, m0:m0+r, tile] (one box of exactly r rows,
-//     from the tensor map whose box height is r); rows m >= n_i are never requested (the
-//     abandoned mini-batches of Alg. 1 cost no bandwidth);
-//   * T/4 consumer threads wait on a slot's "full" barrier, sum the rows in fp32 (m ascending),
-//     apply normalisation + momentum + mix + update with the same operation sequence as the
-//     direct-load kernels (bit-identical results), store x_i and v_i with 128-bit stores and hand
-//     the slot back through its "empty" barrier.
+//   * an X producer thread brings the K old model rows X[:, tile] into a double-buffered X stage
+//     with one box copy per tile (the mix needs every neighbour's OLD value while X is updated in
+//     place); tile t+1's models load while tile t is consumed;
+//   * the consumers form NG groups of T/4 threads; group g owns the learners i = g, g+NG, ...
+//     (their updates are independent once the old models are staged) and a PRIVATE ring of slots;
+//     its own producer thread streams that group's "items" into the ring: item = momentum row
+//     V[i, tile] (one box) + up to R finished gradient rows G[i, m0:m0+r, tile] (one box of exactly
+//     r rows, from the tensor map whose box height is r); rows m >= n_i are never requested (the
+//     abandoned mini-batches of Alg. 1 cost no bandwidth).  A slot is always filled for and released
+//     by the same group, in order: that is what makes waiting on a phase parity unambiguous, and a
+//     slow group never holds up another group's copies;
+//   * a consumer thread owns 4 columns: it waits on the slot's "full" barrier, sums the rows in
+//     fp32 (m ascending), applies normalisation + momentum + mix + update with the same operation
+//     sequence as the direct-load kernels (bit-identical results), stores x_i and v_i with 128-bit
+//     stores and hands the slot back through its "empty" barrier.
 //
 // No CTA ever waits on another CTA.  Every mbarrier wait is bounded: after ~1 s of cycles a
 // waiting thread records an error code in global memory, all roles drain and the kernel returns
@@ -142,7 +148,7 @@ __host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, i
 
 // ES = bytes per gradient element (2: bf16, 4: fp32).
 template <int ES, bool MEAN>
-__global__ void __launch_bounds__(32 + 512, 1) nb_step_pipeline_kernel(const __grid_constant__ PipeArgs a) {
+__global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeline_kernel(const __grid_constant__ PipeArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
   const StepArgs &s = a.s;
@@ -191,60 +197,53 @@ __global__ void __launch_bounds__(32 + 512, 1) nb_step_pipeline_kernel(const __g
   const int64_t ldx = s.ldx;
   bool ok = true;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ producer (one thread)
+  if (warp < NG) {
+    // ------------------------------------------- item producers: one thread per consumer group
+    // Producer g (lane 0 of warp g) feeds group g's private ring with the items of the learners
+    // i = g, g+NG, ... ; a slot is always filled for, and released by, the same group, in order,
+    // which is what makes waiting on a phase parity unambiguous, and a slow group never holds up
+    // the copies of another.
     if (lane == 0) {
-      // Every consumer group has a private ring of NSG slots (items of learner i go to ring i % NG):
-      // a slot is then always filled for, and released by, the same group, in order, which is
-      // what makes waiting on a phase parity unambiguous.
-      uint32_t ring_slot = 0;   // 8 bits per group: next slot of that group's ring
-      uint32_t ring_phase = 0;  // 1 bit per group: phase parity of that ring
-      int titer = 0;
-      // X stage b = titer & 1 is reused every second tile; its k-th use waits for the (k-1)-th release
-      auto issue_x = [&](int tile_x, int it_x) -> bool {
-        const int b = it_x & 1;
-        if (!mbar_wait(&xempty[b], ((it_x >> 1) & 1) ^ 1, a.err, 1)) return false;
-        mbar_expect_tx(&xfull[b], (uint32_t)(K * T * 4));
-        tma_load_2d(xs_base + (size_t)b * K * T, &a.xmap, tile_x * kBoxInner, 0, &xfull[b]);
-        return true;
-      };
-      if (blockIdx.x < a.n_tiles) ok = issue_x(blockIdx.x, 0);
-      for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x, ++titer) {
+      const int g = warp;
+      uint32_t slot = 0, phase = 0;
+      for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x) {
         const int c0 = tile * kBoxInner;  // the tile's first unit in every map
-        const bool have_next = tile + (int)gridDim.x < a.n_tiles;
-        int g = 0;  // i % NG
-        for (int i = 0; ok && i < K; ++i, g = (g + 1 == NG) ? 0 : g + 1) {
-          // the next tile's models are requested half-way through this tile: late enough that the
-          // stage they replace (tile t-1's) has been released, early enough to hide the latency
-          if (have_next && i == K / 2 && !(ok = issue_x(tile + gridDim.x, titer + 1))) break;
+        for (int i = g; ok && i < K; i += NG) {
           const int n = s.n[i];
           int m0 = 0;
           do {
             const int rows = (n - m0 < R) ? (n - m0) : R;
-            const uint32_t gs = (ring_slot >> (8 * g)) & 0xFFu;
-            const uint32_t sl = (uint32_t)g * NSG + gs;
-            if (!(ok = mbar_wait(&empty[sl], ((ring_phase >> g) & 1u) ^ 1u, a.err, 2))) break;
+            const uint32_t sl = (uint32_t)g * NSG + slot;
+            if (!(ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2))) break;
             unsigned char *dst = slots + (size_t)sl * L.slot_bytes;
             const uint32_t bytes = (uint32_t)(rows * T * ES + (m0 == 0 ? T * 4 : 0));
             mbar_expect_tx(&full[sl], bytes);
             if (m0 == 0) tma_load_2d(dst, &a.vmap, c0, i, &full[sl]);
             if (rows > 0) tma_load_3d(dst + T * 4, &a.gmap[rows - 1], c0, m0, i, &full[sl]);
-            if (gs + 1 == (uint32_t)NSG) {
-              ring_slot &= ~(0xFFu << (8 * g));
-              ring_phase ^= 1u << g;
-            } else {
-              ring_slot += 1u << (8 * g);
-            }
+            if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
             m0 += R;
           } while (m0 < n);
         }
+      }
+    }
+  } else if (warp == NG) {
+    // ------------------------------------------- X producer: the tiles' old models, two stages
+    // Stage b = titer & 1 is reused every second tile; its k-th use waits for the (k-1)-th release,
+    // so tile t+1's models load while tile t is consumed.
+    if (lane == 0) {
+      int titer = 0;
+      for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x, ++titer) {
+        const int b = titer & 1;
+        if (!(ok = mbar_wait(&xempty[b], ((titer >> 1) & 1) ^ 1, a.err, 1))) break;
+        mbar_expect_tx(&xfull[b], (uint32_t)(K * T * 4));
+        tma_load_2d(xs_base + (size_t)b * K * T, &a.xmap, tile * kBoxInner, 0, &xfull[b]);
       }
     }
   } else {
     // ------------------------------------------------- consumers: NG groups of T/4 threads each
     // Group g owns the learners i with i % NG == g (their updates are independent of each other
     // once the old models are staged), so several ring items are consumed concurrently.
-    const int ct = threadIdx.x - 32;
+    const int ct = threadIdx.x - 32 * (NG + 1);
     const int nq = T / 4;  // float4 per staged row = threads per group
     const int grp = ct / nq, cq = ct - grp * nq;
     {
@@ -413,28 +412,33 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   if (R < 1) R = 1;
   if (R > kMaxRowsPerItem) R = kMaxRowsPerItem;
   if (R > a.M) R = a.M;
-  // Tile width: a box row is 256 units of T*es/256 bytes, so T is 128, 256 or 512.  CTAs per SM and
-  // T shrink until the ring has at least 3 slots beside the double-buffered X stage.
-  int T = t.T ? t.T : 512;
-  int ctas = t.ctas_per_sm ? t.ctas_per_sm : 2;
-  int groups = 1, slots = 0;
-  for (;;) {
+  // Tile width: a box row is 256 units of T*es/256 bytes, so T is 128, 256 or 512.
+  // Shapes tried in order (measured on B200, see profiles/): two CTAs per SM with two consumer
+  // groups each while the double-buffered X stage leaves room for it (K <= 16 at T = 512), else one
+  // CTA per SM with four groups; then narrower tiles.  The first shape whose ring has at least two
+  // slots per group is taken.  Environment overrides replace the corresponding field of every shape.
+  struct Shape { int T, ctas, groups; };
+  const Shape shapes[] = {{512, 2, 2}, {512, 1, 4}, {256, 1, 4}, {128, 1, 4}};
+  int T = 0, ctas = 0, groups = 0, slots = 0;
+  bool found = false;
+  for (const Shape &sh : shapes) {
+    T = t.T ? t.T : sh.T;
+    ctas = t.ctas_per_sm ? t.ctas_per_sm : sh.ctas;
+    groups = t.groups ? t.groups : sh.groups;
     if (T != 128 && T != 256 && T != 512) return false;
-    groups = t.groups ? t.groups : 2;
     if (groups > kMaxGroups) groups = kMaxGroups;
     if (groups > a.K) groups = a.K;
     while (groups > 1 && groups * (T / 4) > 512) --groups;
+    if (groups < 1 || ctas < 1) return false;
     const PipeLayout L0 = pipe_layout(a.K, T, es, R, 0, a.mix_slots);
     const int budget = kSmemBudget / ctas - 1024;
     slots = (budget - L0.total - 256) / (T * 4 + R * T * es);
     if (t.slots && t.slots < slots) slots = t.slots;
     if (slots > 32) slots = 32;
     slots -= slots % groups;  // every group's ring has the same number of slots
-    if (slots >= 2 * groups) break;
-    if (ctas > 1 && !t.ctas_per_sm) { --ctas; continue; }
-    if (T > 128 && !t.T) { T /= 2; continue; }
-    return false;
+    if (slots >= 2 * groups) { found = true; break; }
   }
+  if (!found) return false;
   if (a.P < T) return false;
   const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots);
   if (L.total > kSmemBudget) return false;
@@ -490,7 +494,7 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
       if (!encode_map(&p.gmap[r - 1], a.G, ub, 3, dims, strides, box)) return cudaErrorInvalidValue;
     }
   }
-  const int threads = 32 + plan.n_groups * (plan.T / 4);
+  const int threads = 32 + plan.n_groups * (32 + plan.T / 4);  // X producer + per group: producer warp + consumers
   if (es == 2) {
     if (a.mean_mode) nb_step_pipeline_kernel<2, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
     else nb_step_pipeline_kernel<2, false><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
