@@ -243,6 +243,7 @@ def run_ours(args, w):
     e1.record()
     barrier()
     clocks = sampler.stop()
+    kernel_plan = ctx.get_kernel_plan()
     launches = ctx.get_stats()["kernel_launches"] - launches0
     total_ms = e0.elapsed_time(e1)
     launch_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
@@ -257,7 +258,8 @@ def run_ours(args, w):
                 "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_per_launch) if TRAFFIC_PER_ALGORITHMIC_BYTE else None,
                 "peak_source": "of " + peak_kind, "kernel": "nb_step_pipeline_kernel (fused accumulate+mix+momentum+update)",
                 "algorithmic_bytes_per_launch": bytes_per_launch, "launch_ms": launch_ms,
-                "frac_of_8TBps_nominal": achieved / 8000.0, "mean_sum_finished": sum_n / args.steps}
+                "frac_of_8TBps_nominal": achieved / 8000.0, "mean_sum_finished": sum_n / args.steps,
+                "kernel_plan": kernel_plan}
 
     # ---- end to end: host gradient buffers through nb_step_fused_host -------------------------
     e2e = None

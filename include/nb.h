@@ -255,6 +255,13 @@ int nb_get_device_mixing(nb_ctx *c, uint32_t *bits, float *W_dense, void *stream
 int nb_get_stats(const nb_ctx *c, int64_t *sum_finished, double *algorithmic_bytes,
                  int64_t *kernel_launches);
 
+/* Which kernel shape ran the most recent step (for reports and tests), host out plan[8]:
+ * [0] 1 if the bulk-copy pipeline kernel covered the full tiles, 0 if the direct-load kernel did
+ * everything; [1] tile width in columns; [2] consumer groups per CTA; [3] ring slots per CTA;
+ * [4] gradient rows per ring item; [5] CTAs launched; [6] dynamic shared memory per CTA in bytes;
+ * [7] tiles covered (columns beyond [7]*[1] went to the direct-load kernel). */
+int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan);
+
 /* ------------------------------------------------------------------------------------------------
  * Allocation-free variant (no counterpart in the paper: it exists for deployment reasons only).
  *

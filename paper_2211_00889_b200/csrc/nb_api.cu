@@ -30,6 +30,7 @@ struct nb_ctx {
   int acc_esize = 4;
   int64_t sum_finished = 0, launches = 0;
   double alg_bytes = 0.0;
+  nb::PipePlan last_plan{};  // shape of the pipeline kernel of the most recent step (zeros: not used)
   int sticky = NB_OK;
   std::string err;
 };
@@ -179,7 +180,7 @@ int run_update(nb_ctx *c, nb::StepArgs *a, int src, cudaStream_t st) {
     int rc = build_device_mixing(c, st);
     if (rc != NB_OK) return rc;
     int n_launched = 0;
-    cudaError_t e = nb::launch_step(*a, src, c->d_err, &n_launched, st);
+    cudaError_t e = nb::launch_step(*a, src, c->d_err, &n_launched, &c->last_plan, st);
     c->launches += n_launched;
     if (e != cudaSuccess) return cuda_fail(c, e, "launch_step");
   }
@@ -560,6 +561,20 @@ int nb_get_device_mixing(nb_ctx *c, uint32_t *bits, float *W_dense, void *stream
         if (e2 >= 0 && e2 < NB_MAX_NNZ && h->col[e2] >= 0 && h->col[e2] < K) W_dense[(size_t)i * K + h->col[e2]] += h->val[e2];
   }
   delete h;
+  return NB_OK;
+}
+
+int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan) {
+  if (!c || !plan) return NB_ERR_ARG;
+  const nb::PipePlan &p = c->last_plan;
+  plan[0] = p.n_tiles > 0 ? 1 : 0;
+  plan[1] = p.T;
+  plan[2] = p.n_groups;
+  plan[3] = p.n_slots;
+  plan[4] = p.rows_per_item;
+  plan[5] = p.grid;
+  plan[6] = p.smem_bytes;
+  plan[7] = p.n_tiles;
   return NB_OK;
 }
 

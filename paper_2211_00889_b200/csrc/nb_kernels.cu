@@ -287,8 +287,9 @@ static cudaError_t launch_step_direct(const StepArgs &a, int src, cudaStream_t s
 
 cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st) { return launch_step_direct(a, src, st); }
 
-cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st) {
+cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, PipePlan *used, cudaStream_t st) {
   *launches = 0;
+  *used = PipePlan{};
   // The pipeline kernel sees one gradient-like stream; the unfused step presents the accumulator
   // as a one-row fp32 stream (0 + acc == acc bit for bit: acc is never -0).
   StepArgs p = a;
@@ -306,6 +307,7 @@ cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches
     cudaError_t e = launch_step_pipeline(p, es, plan, err_flag, st);
     if (e != cudaSuccess) return e;
     ++*launches;
+    *used = plan;
     done = (int64_t)plan.n_tiles * plan.T;
   }
   if (done < a.P) {  // ragged tail (or everything, when the pipeline does not apply)

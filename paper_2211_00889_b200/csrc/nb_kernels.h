@@ -51,7 +51,7 @@ struct MatchaArgs {
 
 // Bulk-copy pipeline kernel (nb_pipeline.cu)
 struct PipePlan {
-  int T, rows_per_item, n_slots, n_groups, smem_bytes, n_tiles, grid;
+  int T, rows_per_item, n_slots, n_groups, smem_bytes, n_tiles, grid;  // all 0: the pipeline kernel did not run
 };
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan);
 cudaError_t configure_pipeline();
@@ -61,7 +61,7 @@ int step_threads_per_block(const StepArgs &a);
 cudaError_t launch_accumulate(const StepArgs &a, int src, cudaStream_t st);
 // Runs the step on all P columns: pipeline kernel on the full tiles when it applies, direct-load
 // kernel on the rest.  *launches receives the number of kernels launched.
-cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st);
+cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, PipePlan *used, cudaStream_t st);
 // The direct-load step kernel on all P columns (no pipeline kernel, no device error word).
 cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st);
 cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,

@@ -50,3 +50,17 @@ def test_argument_errors_are_reported_without_a_gpu():
     assert h.value is None
     assert B.lib.nb_destroy(None) == B.NB_OK
     assert B.lib.nb_step(None, None) == B.NB_ERR_ARG
+
+
+def test_valid_create_fails_loudly_without_a_gpu():
+    import torch
+    if torch.cuda.is_available():
+        import pytest
+        pytest.skip("a CUDA device is present")
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    h = ctypes.c_void_p()
+    rc = B.lib.nb_create(ctypes.byref(h), 4, 1024, 4, 0.1, 0.9, B.NB_ALLREDUCE, None)
+    assert rc in (B.NB_ERR_CUDA, B.NB_ERR_NOMEM) and h.value is None      # no CPU fallback exists
+    assert B.lib.nb_last_error(None) != b""

@@ -60,6 +60,20 @@ def test_sizes_around_one_tile(B, P, expected_launches):
     assert launches == [expected_launches] * w.steps
 
 
+def test_bench_workload_runs_on_the_pipeline_kernel(B):
+    """The shape the planner picks for the benchmark workload (a narrow slice of it is enough)."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 8 * 512, steps=1)
+    ctx = B.context_for(w)
+    ctx.set_params(torch.from_numpy(WL.init_params(w)).cuda())
+    assert ctx.get_kernel_plan()["pipeline"] == 0                      # nothing has run yet
+    ctx.step_fused(H.to_device(WL.gradients_np(w, 0)[0]), H.lib_counts(B, w, 0))
+    plan = ctx.get_kernel_plan()
+    assert plan["pipeline"] == 1 and plan["tile"] == 512 and plan["tiles"] == 8
+    assert plan["groups"] >= 1 and plan["slots"] >= 2 * plan["groups"] and plan["smem_bytes"] <= 227 * 1024
+    ctx.close()
+
+
 @pytest.mark.parametrize("K", [2, 3, 17, 33, 64])
 @pytest.mark.parametrize("variant", ["dpsgd", "allreduce"])
 def test_learner_counts(B, K, variant):
