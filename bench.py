@@ -47,6 +47,10 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", default="", choices=["", "allreduce", "dpsgd", "centralized"],
+                    help="run the workload's sizes with another variant (dpsgd = ring)")
+    ap.add_argument("--order", default="mix_then_update", choices=["mix_then_update", "update_then_mix"])
+    ap.add_argument("--unfused", action="store_true", help="time nb_accumulate + nb_step instead of nb_step_fused")
     ap.add_argument("--cols", type=int, default=0, help="profiling aid: run the workload on this many columns instead of its P")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
@@ -130,7 +134,8 @@ def time_oracle(w, sample_cols, steps, warmup=0):
     from oracle import nb_oracle as O
     from paper_2211_00889_b200 import workloads as WL
     ws = WL.scaled(w, min(sample_cols, w.P))
-    if w.variant == "allreduce":
+    central = w.variant == "centralized"
+    if w.variant in ("allreduce", "centralized"):
         orc = O.Oracle(ws.K, ws.P, ws.M, ws.lr, ws.mom, "allreduce")
     elif w.variant == "dpsgd":
         orc = O.Oracle(ws.K, ws.P, ws.M, ws.lr, ws.mom, "dpsgd", W=O.ring_W(ws.K))
@@ -138,13 +143,18 @@ def time_oracle(w, sample_cols, steps, warmup=0):
         partner = O.greedy_matchings(O.random_regular_graph(ws.seed, ws.K, ws.degree)[0], ws.K)
         orc = O.Oracle(ws.K, ws.P, ws.M, ws.lr, ws.mom, "matcha", partner=partner, alpha=ws.alpha,
                        prob=ws.act_prob, seed=ws.seed)
-    orc.set_params(WL.init_params(ws))
+    x0 = WL.init_params(ws)
+    orc.set_params(x0)
+    x_ps, v_ps = x0.astype(np.float64), np.zeros(ws.P)
     G = WL.gradients_torch(ws, 0, "cpu").float().numpy()     # one block, reused (not timed)
     total = 0.0
     for t in range(warmup + steps):
         n = O.straggler_counts(ws.straggler_model, ws.seed, t, ws.K, ws.M, ws.straggler_params)
         t0 = time.perf_counter()
-        orc.step(G, n)
+        if central:
+            x_ps, v_ps = O.step_centralized(x_ps, v_ps, G, n, ws.lr, ws.mom)
+        else:
+            orc.step(G, n)
         dt = time.perf_counter() - t0
         if t >= warmup:
             total += dt
@@ -213,13 +223,22 @@ def run_ours(args, w):
     x0 = torch.randn(w.P, generator=gen, device=dev, dtype=torch.float32) * w.init_sigma
     ctx = B.context_for(w)
     ctx.set_params(x0)
+    if args.order == "update_then_mix":
+        ctx.set_option(B.NB_OPT_ORDER, B.NB_ORDER_UPDATE_THEN_MIX)
+
+    def one_step(g, n):
+        if args.unfused:
+            ctx.accumulate(g, n)
+            ctx.step()
+        else:
+            ctx.step_fused(g, n)
 
     def counts(t):
         return B.straggler_sample(w.straggler_model, w.seed, t, w.K, w.M, w.straggler_params)[0]
 
     total_steps = args.warmup + args.steps
     for t in range(args.warmup):
-        ctx.step_fused(bufs[t % n_buf], counts(t))
+        one_step(bufs[t % n_buf], counts(t))
     if world > 1:   # every rank derives the counts by itself; they must coincide (checked outside the timed region)
         assert sharding.counts_agree(counts(args.warmup), dev), "ranks disagree on the finished counts"
     barrier()
@@ -235,7 +254,7 @@ def run_ours(args, w):
         t = args.warmup + s
         n = counts(t)                      # S0: host straggler simulator, inside the timed step
         ev[s][0].record()
-        ctx.step_fused(bufs[t % n_buf], n)
+        one_step(bufs[t % n_buf], n)
         ev[s][1].record()
         st = ctx.get_stats()
         alg_bytes += st["algorithmic_bytes"]
@@ -301,7 +320,9 @@ def run_ours(args, w):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "K": w.K, "P": w.P, "M": w.M, "grad_dtype": w.grad_dtype,
-                       "variant": w.variant, "topology": w.topology, "parallelism": "column-shard x%d" % world,
+                       "variant": w.variant, "topology": w.topology, "order": args.order,
+                       "entry": "nb_accumulate+nb_step" if args.unfused else "nb_step_fused",
+                       "parallelism": "column-shard x%d" % world,
                        "l2": "inputs larger than L2 (%.1f GB gradient stream x%d buffers + %.1f GB state per step)"
                              % (g_bytes / 1e9, n_buf, 2 * w.K * w.P * 4 / 1e9)},
             "achieved_hbm_gbs": achieved, "frac_of_8TBps": achieved / 8000.0,
@@ -320,6 +341,10 @@ def main():
     if args.cols:
         from dataclasses import replace
         w = replace(WL.scaled(w, args.cols), name="%s[P=%d]" % (w.name, args.cols))
+    if args.variant:
+        from dataclasses import replace
+        topo = {"allreduce": "full", "dpsgd": "ring", "centralized": "full"}[args.variant]
+        w = replace(w, variant=args.variant, topology=topo, name="%s[%s]" % (w.name, args.variant))
     if args.impl == "reference":
         run_reference(args, w)
     else:

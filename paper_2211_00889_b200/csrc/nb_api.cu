@@ -174,8 +174,10 @@ int build_device_mixing(nb_ctx *c, cudaStream_t st) {
 int run_update(nb_ctx *c, nb::StepArgs *a, int src, cudaStream_t st) {
   fill_update_args(c, a);
   if (c->variant == NB_CENTRALIZED) {
-    NB_CUDA(c, nb::launch_centralized(*a, src, st));
-    c->launches++;
+    int n_launched = 0;
+    cudaError_t e = nb::launch_centralized(*a, src, c->d_err, &n_launched, st);
+    c->launches += n_launched;
+    if (e != cudaSuccess) return cuda_fail(c, e, "launch_centralized");
   } else {
     int rc = build_device_mixing(c, st);
     if (rc != NB_OK) return rc;
@@ -355,8 +357,11 @@ int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t
   int es = 4;
   int rc = fill_step_args(c, grads, dtype, ld_m, ld_k, finished, &a, &es);
   if (rc != NB_OK) return rc;
-  NB_CUDA(c, nb::launch_accumulate(a, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16, (cudaStream_t)stream));
-  c->launches++;
+  int n_launched = 0;
+  cudaError_t e = nb::launch_accumulate(a, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16, c->d_err, &n_launched,
+                                        (cudaStream_t)stream);
+  c->launches += n_launched;
+  if (e != cudaSuccess) return cuda_fail(c, e, "launch_accumulate");
   std::memcpy(c->n_acc, a.n, sizeof(c->n_acc));
   c->acc_esize = es;
   c->acc_fresh = true;

@@ -265,7 +265,50 @@ cudaError_t configure_kernels() {
   return configure_pipeline();
 }
 
-cudaError_t launch_accumulate(const StepArgs &a, int src, cudaStream_t st) {
+namespace {
+// Column range [done, P) of the same problem: what the direct-load kernels take over after a
+// pipeline kernel has covered the full tiles.
+StepArgs tail_of(const StepArgs &a, int64_t done, int es) {
+  StepArgs r = a;
+  r.X += done;
+  r.V += done;
+  r.acc += done;
+  r.G = reinterpret_cast<const unsigned char *>(a.G) + done * es;
+  r.P = a.P - done;
+  return r;
+}
+// The accumulator presented as a one-row fp32 gradient stream (0 + acc == acc bit for bit: acc is never -0).
+StepArgs acc_as_stream(const StepArgs &a) {
+  StepArgs p = a;
+  p.G = a.acc;
+  p.ld_m = a.ldx;
+  p.ld_k = a.ldx;
+  p.M = 1;
+  for (int i = 0; i < a.K; ++i) p.n[i] = 1;
+  return p;
+}
+}  // namespace
+
+cudaError_t launch_accumulate(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st) {
+  *launches = 0;
+  const int es = src == kSrcBF16 ? 2 : 4;
+  PipePlan plan;
+  int64_t done = 0;
+  if (plan_stream(a, es, false, &plan)) {
+    cudaError_t e = launch_stream_pipeline(a, es, false, plan, err_flag, st);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+    done = (int64_t)plan.n_tiles * plan.T;
+  }
+  if (done < a.P) {
+    cudaError_t e = launch_accumulate_direct_only(tail_of(a, done, es), src, st);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  return cudaSuccess;
+}
+
+cudaError_t launch_accumulate_direct_only(const StepArgs &a, int src, cudaStream_t st) {
   const int tpb = 256;
   const int64_t per_block = (int64_t)tpb * kColsPerThread;
   dim3 grid((unsigned)((a.P + per_block - 1) / per_block), (unsigned)a.K);
@@ -290,17 +333,9 @@ cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st)
 cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, PipePlan *used, cudaStream_t st) {
   *launches = 0;
   *used = PipePlan{};
-  // The pipeline kernel sees one gradient-like stream; the unfused step presents the accumulator
-  // as a one-row fp32 stream (0 + acc == acc bit for bit: acc is never -0).
-  StepArgs p = a;
-  int es = src == kSrcBF16 ? 2 : 4;
-  if (src == kSrcAcc) {
-    p.G = a.acc;
-    p.ld_m = a.ldx;
-    p.ld_k = a.ldx;
-    p.M = 1;
-    for (int i = 0; i < a.K; ++i) p.n[i] = 1;
-  }
+  // The pipeline kernel sees one gradient-like stream; the unfused step presents the accumulator as one.
+  const int es = src == kSrcBF16 ? 2 : 4;
+  const StepArgs p = src == kSrcAcc ? acc_as_stream(a) : a;
   PipePlan plan;
   int64_t done = 0;
   if (plan_pipeline(p, es, &plan)) {
@@ -311,13 +346,7 @@ cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches
     done = (int64_t)plan.n_tiles * plan.T;
   }
   if (done < a.P) {  // ragged tail (or everything, when the pipeline does not apply)
-    StepArgs r = a;
-    r.X += done;
-    r.V += done;
-    r.acc += done;
-    r.G = reinterpret_cast<const unsigned char *>(a.G) + done * es;
-    r.P = a.P - done;
-    cudaError_t e = launch_step_direct(r, src, st);
+    cudaError_t e = launch_step_direct(tail_of(a, done, es), src, st);
     if (e != cudaSuccess) return e;
     ++*launches;
   }
@@ -337,7 +366,29 @@ cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool al
   return cudaGetLastError();
 }
 
-cudaError_t launch_centralized(const StepArgs &a, int src, cudaStream_t st) {
+static cudaError_t launch_centralized_direct(const StepArgs &a, int src, cudaStream_t st);
+
+cudaError_t launch_centralized(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st) {
+  *launches = 0;
+  const int es = src == kSrcBF16 ? 2 : 4;
+  const StepArgs p = src == kSrcAcc ? acc_as_stream(a) : a;
+  PipePlan plan;
+  int64_t done = 0;
+  if (plan_stream(p, es, true, &plan)) {
+    cudaError_t e = launch_stream_pipeline(p, es, true, plan, err_flag, st);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+    done = (int64_t)plan.n_tiles * plan.T;
+  }
+  if (done < a.P) {
+    cudaError_t e = launch_centralized_direct(tail_of(a, done, es), src, st);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  return cudaSuccess;
+}
+
+static cudaError_t launch_centralized_direct(const StepArgs &a, int src, cudaStream_t st) {
   const int tpb = 256;
   const int64_t per_block = (int64_t)tpb * kColsPerThread;
   const unsigned grid = (unsigned)((a.P + per_block - 1) / per_block);

@@ -54,11 +54,16 @@ struct PipePlan {
   int T, rows_per_item, n_slots, n_groups, smem_bytes, n_tiles, grid;  // all 0: the pipeline kernel did not run
 };
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan);
+bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan);
+cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, const PipePlan &plan, int *err_flag,
+                                   cudaStream_t st);
 cudaError_t configure_pipeline();
 cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan, int *err_flag, cudaStream_t st);
 
 int step_threads_per_block(const StepArgs &a);
-cudaError_t launch_accumulate(const StepArgs &a, int src, cudaStream_t st);
+// Masked accumulate on all P columns (pipeline kernel on the full tiles when it applies).
+cudaError_t launch_accumulate(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st);
+cudaError_t launch_accumulate_direct_only(const StepArgs &a, int src, cudaStream_t st);
 // Runs the step on all P columns: pipeline kernel on the full tiles when it applies, direct-load
 // kernel on the rest.  *launches receives the number of kernels launched.
 cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, PipePlan *used, cudaStream_t st);
@@ -66,7 +71,7 @@ cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches
 cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st);
 cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,
                                  cudaStream_t st);
-cudaError_t launch_centralized(const StepArgs &a, int src, cudaStream_t st);
+cudaError_t launch_centralized(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st);
 cudaError_t launch_matcha_build(const MatchaArgs &a, cudaStream_t st);
 cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, cudaStream_t st);
 cudaError_t configure_kernels();

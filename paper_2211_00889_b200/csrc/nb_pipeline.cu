@@ -329,6 +329,129 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
   if (!ok) drain_and_exit_delay();
 }
 
+// -------------------------------------------------------------------------------------------------
+// The same producer / ring machinery for the two steps that need no X stage:
+//   kModeAccumulate : acc[i, tile] = sum_{m < n_i} G[i, m, tile]              (nb_accumulate)
+//   kModeCentralized: g = (1/K) sum_i s_i acc_i; v <- mom v + g; x <- x - lr v  (Alg. 3, one model)
+// Items carry gradient rows only.  Accumulate uses NG groups (learners are independent); the
+// centralized step uses one group so that the learners are folded in ascending order, exactly as
+// the direct-load kernel does.
+// -------------------------------------------------------------------------------------------------
+constexpr int kModeAccumulate = 0, kModeCentralized = 1;
+
+struct StreamLayout {
+  int32_t off_slots, slot_bytes, total;
+};
+__host__ __device__ inline StreamLayout stream_layout(int T, int es, int R, int n_slots) {
+  StreamLayout L;
+  int off = 2 * n_slots * 8;
+  off = (off + 127) / 128 * 128;
+  L.off_slots = off;
+  L.slot_bytes = R * T * es;
+  L.total = off + n_slots * L.slot_bytes;
+  return L;
+}
+
+template <int ES, int MODE>
+__global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline_kernel(const __grid_constant__ PipeArgs a) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
+  const StepArgs &s = a.s;
+  const int K = s.K, T = a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
+  const int NSG = NS / NG;
+  const StreamLayout L = stream_layout(T, ES, R, NS);
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);
+  uint64_t *empty = full + NS;
+  unsigned char *slots = smem_raw + L.off_slots;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int group_warps = T / 128;
+  if (threadIdx.x == 0) {
+    for (int q = 0; q < NS; ++q) {
+      mbar_init(&full[q], 1);
+      mbar_init(&empty[q], group_warps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const int64_t ldx = s.ldx;
+  bool ok = true;
+
+  if (warp < NG) {
+    if (lane == 0) {  // producer of group `warp`
+      const int g = warp;
+      uint32_t slot = 0, phase = 0;
+      for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x) {
+        const int c0 = tile * kBoxInner;
+        for (int i = g; ok && i < K; i += NG) {
+          const int n = s.n[i];
+          int m0 = 0;
+          do {
+            const int rows = (n - m0 < R) ? (n - m0) : R;
+            const uint32_t sl = (uint32_t)g * NSG + slot;
+            if (!(ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2))) break;
+            mbar_expect_tx(&full[sl], (uint32_t)(rows * T * ES));  // 0 rows: a plain arrival
+            if (rows > 0) tma_load_3d(slots + (size_t)sl * L.slot_bytes, &a.gmap[rows - 1], c0, m0, i, &full[sl]);
+            if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
+            m0 += R;
+          } while (m0 < n);
+        }
+      }
+    }
+  } else {
+    const int ct = threadIdx.x - 32 * NG;
+    const int nq = T / 4;
+    const int grp = ct / nq, cq = ct - grp * nq;
+    uint32_t slot = 0, phase = 0;
+    for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x) {
+      const int64_t col0 = (int64_t)tile * T + (int64_t)cq * 4;
+      float4 x = make_float4(0.f, 0.f, 0.f, 0.f), v = x, gs = x;
+      if constexpr (MODE == kModeCentralized) {  // requested early, used after the last learner
+        x = ld4(s.X + col0);
+        v = ld4(s.V + col0);
+      }
+      for (int i = grp; ok && i < K; i += NG) {
+        const int n = s.n[i];
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        int m0 = 0;
+        do {
+          const int rows = (n - m0 < R) ? (n - m0) : R;
+          const uint32_t sl = (uint32_t)grp * NSG + slot;
+          ok = __all_sync(0xffffffffu, mbar_wait(&full[sl], phase, a.err, 4));
+          if (!ok) break;
+          const unsigned char *rowp = slots + (size_t)sl * L.slot_bytes + (size_t)cq * 4 * ES;
+          for (int r = 0; r < rows; ++r) {
+            Raw<SRC> raw;
+            if constexpr (ES == 2) raw.r = *reinterpret_cast<const uint2 *>(rowp + (size_t)r * T * ES);
+            else raw.r = *reinterpret_cast<const float4 *>(rowp + (size_t)r * T * ES);
+            acc = add4(acc, widen(raw));
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&empty[sl]);
+          if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
+          m0 += R;
+        } while (m0 < n);
+        if (!ok) break;
+        if constexpr (MODE == kModeAccumulate) {
+          st4(s.acc + (int64_t)i * ldx + col0, acc);
+        } else {
+          const float si = s.s[i];
+          gs.x = __fmaf_rn(si, acc.x, gs.x);
+          gs.y = __fmaf_rn(si, acc.y, gs.y);
+          gs.z = __fmaf_rn(si, acc.z, gs.z);
+          gs.w = __fmaf_rn(si, acc.w, gs.w);
+        }
+      }
+      if (!ok) break;
+      if constexpr (MODE == kModeCentralized) {
+        const float4 vn = momentum(s.mom, v, s.inv_K, gs);
+        st4(s.V + col0, vn);
+        st4(s.X + col0, descend(x, s.lr, vn));
+      }
+    }
+  }
+  if (!ok) drain_and_exit_delay();
+}
+
 struct PipeTuning {
   int enabled = 1, T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0;
   int sm_count = 0;
@@ -453,6 +576,78 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   return plan->n_tiles > 0;
 }
 
+// Shape of the no-stage kernel: T = 512 (or narrower), R rows per item, as many CTAs per SM as
+// keep at least 3 slots per group.
+bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
+  PipeTuning &t = tuning();
+  if (!t.enabled) return false;
+  if (t.sm_count == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&t.sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (t.sm_count <= 0) t.sm_count = 148;
+  }
+  if ((uintptr_t)a.G % 16 != 0 || (a.ld_m * es) % 16 != 0 || (a.ld_k * es) % 16 != 0) return false;
+  if (!encode_fn()) return false;
+  const int T = 512;
+  if (a.P < T) return false;
+  int R = es == 2 ? 8 : 4;
+  if (R > a.M) R = a.M;
+  int groups = centralized ? 1 : 2;
+  if (groups > a.K) groups = a.K;
+  const int ctas = centralized ? 4 : 2;
+  const int budget = kSmemBudget / ctas - 1024;
+  int slots = (budget - 512) / (R * T * es);
+  if (slots > 16) slots = 16;
+  slots -= slots % groups;
+  if (slots < 2 * groups) return false;
+  plan->T = T;
+  plan->rows_per_item = R;
+  plan->n_slots = slots;
+  plan->n_groups = groups;
+  plan->smem_bytes = stream_layout(T, es, R, slots).total;
+  plan->n_tiles = (int)(a.P / T);
+  const int64_t max_ctas = (int64_t)ctas * t.sm_count;
+  plan->grid = (int)(plan->n_tiles < max_ctas ? plan->n_tiles : max_ctas);
+  return plan->n_tiles > 0;
+}
+
+bool encode_gmaps(PipeArgs *p, const StepArgs &a, int es, const PipePlan &plan) {
+  const cuuint64_t units = (cuuint64_t)plan.n_tiles * kBoxInner;
+  const int ub = plan.T * es / kBoxInner;
+  const cuuint64_t dims[3] = {units, (cuuint64_t)a.M, (cuuint64_t)a.K};
+  const cuuint64_t strides[2] = {(cuuint64_t)a.ld_m * es, (cuuint64_t)a.ld_k * es};
+  const int rmax = plan.rows_per_item < a.M ? plan.rows_per_item : a.M;
+  for (int r = 1; r <= rmax; ++r) {
+    const cuuint32_t box[3] = {kBoxInner, (cuuint32_t)r, 1};
+    if (!encode_map(&p->gmap[r - 1], a.G, ub, 3, dims, strides, box)) return false;
+  }
+  return true;
+}
+
+cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, const PipePlan &plan, int *err_flag,
+                                   cudaStream_t st) {
+  PipeArgs p;
+  std::memset(&p, 0, sizeof(p));
+  p.s = a;
+  p.T = plan.T;
+  p.n_slots = plan.n_slots;
+  p.rows_per_item = plan.rows_per_item;
+  p.n_tiles = plan.n_tiles;
+  p.n_groups = plan.n_groups;
+  p.err = err_flag;
+  if (!encode_gmaps(&p, a, es, plan)) return cudaErrorInvalidValue;
+  const int threads = plan.n_groups * (32 + plan.T / 4);
+  if (es == 2) {
+    if (centralized) nb_stream_pipeline_kernel<2, kModeCentralized><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
+    else nb_stream_pipeline_kernel<2, kModeAccumulate><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
+  } else {
+    if (centralized) nb_stream_pipeline_kernel<4, kModeCentralized><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
+    else nb_stream_pipeline_kernel<4, kModeAccumulate><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
+  }
+  return cudaGetLastError();
+}
+
 cudaError_t configure_pipeline() {
   cudaError_t e;
 #define NB_CFG(ES, MEAN)                                                                              \
@@ -460,6 +655,12 @@ cudaError_t configure_pipeline() {
                                 kSmemBudget)) != cudaSuccess)                                         \
     return e;
   NB_CFG(2, true) NB_CFG(2, false) NB_CFG(4, true) NB_CFG(4, false)
+#undef NB_CFG
+#define NB_CFG(ES, MODE)                                                                                          \
+  if ((e = cudaFuncSetAttribute(nb_stream_pipeline_kernel<ES, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                kSmemBudget)) != cudaSuccess)                                                     \
+    return e;
+  NB_CFG(2, kModeAccumulate) NB_CFG(2, kModeCentralized) NB_CFG(4, kModeAccumulate) NB_CFG(4, kModeCentralized)
 #undef NB_CFG
   return cudaSuccess;
 }
@@ -484,16 +685,7 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
     if (!encode_map(&p.xmap, a.X, ub, 2, dims, strides, xbox) || !encode_map(&p.vmap, a.V, ub, 2, dims, strides, vbox))
       return cudaErrorInvalidValue;
   }
-  {  // G: [K, M, units]; one map per box height
-    const int ub = plan.T * es / kBoxInner;
-    const cuuint64_t dims[3] = {units, (cuuint64_t)a.M, (cuuint64_t)a.K};
-    const cuuint64_t strides[2] = {(cuuint64_t)a.ld_m * es, (cuuint64_t)a.ld_k * es};
-    const int rmax = plan.rows_per_item < a.M ? plan.rows_per_item : a.M;
-    for (int r = 1; r <= rmax; ++r) {
-      const cuuint32_t box[3] = {kBoxInner, (cuuint32_t)r, 1};
-      if (!encode_map(&p.gmap[r - 1], a.G, ub, 3, dims, strides, box)) return cudaErrorInvalidValue;
-    }
-  }
+  if (!encode_gmaps(&p, a, es, plan)) return cudaErrorInvalidValue;  // G: [K, M, units]; one map per box height
   const int threads = 32 + plan.n_groups * (32 + plan.T / 4);  // X producer + per group: producer warp + consumers
   if (es == 2) {
     if (a.mean_mode) nb_step_pipeline_kernel<2, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);

@@ -102,7 +102,7 @@ extern "C" int nb_step_static(int K, int64_t P, int M, float lr, float mom, floa
   cudaStream_t st = (cudaStream_t)stream;
   // the accumulate kernel writes every element of acc[K, 0:round_up(P,4)) that the step kernel reads,
   // so nothing of the previous call's contents survives into this one
-  e = nb::launch_accumulate(a, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16, st);
+  e = nb::launch_accumulate_direct_only(a, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16, st);
   if (e == cudaSuccess) e = nb::launch_step_direct_only(a, nb::kSrcAcc, st);
   if (e != cudaSuccess) return fail(NB_ERR_CUDA, std::string("nb_step_static: launch: ") + cudaGetErrorString(e));
   return NB_OK;
