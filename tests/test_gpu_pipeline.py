@@ -142,3 +142,62 @@ def test_pipeline_and_direct_kernels_agree_bitwise(B, name, order):
     assert torch.equal(a.get_params(), b.get_params())
     assert torch.equal(a.get_momentum(), b.get_momentum())
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("dtype,P", [("bf16", 4 * 512 + 40), ("f32", 3 * 512 + 12), ("bf16", 512)])
+@pytest.mark.parametrize("fused", [True, False])
+def test_centralized_step_on_pipeline_sizes(B, dtype, P, fused):
+    """Alg. 3 through the no-stage pipeline kernel (aligned rows): oracle parity, and the same bits
+    as the direct-load kernel (which a one-element shift of the stream forces)."""
+    import torch
+    K, M = 8, 8
+    rng = np.random.default_rng(11)
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    a = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
+    b = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
+    for c in (a, b):
+        c.set_params(torch.from_numpy(x0).cuda())
+    x, v = x0.astype(np.float64), np.zeros(P)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    for t in range(4):
+        G = (torch.from_numpy(rng.standard_normal((K, M, P)).astype(np.float32)) * 0.01).to(tdt).cuda()
+        n = rng.integers(0, M + 1, K)
+        flat = torch.empty(G.numel() + 1, dtype=tdt, device="cuda")
+        shifted = flat[1:].view_as(G)
+        shifted.copy_(G)
+        if fused:
+            a.step_fused(G, n); b.step_fused(shifted, n)
+        else:
+            a.accumulate(G, n); a.step()
+            b.accumulate(shifted, n); b.step()
+        x, v = O.step_centralized(x, v, G.float().cpu().numpy(), n.tolist(), 0.1, 0.9)
+    H.assert_close(a.get_params().numpy(), x, H.TOL_SAME_INPUT)
+    H.assert_close(a.get_momentum().numpy(), v, H.TOL_SAME_INPUT)
+    assert torch.equal(a.get_params(), b.get_params()) and torch.equal(a.get_momentum(), b.get_momentum())
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("M", [3, 8, 19])
+def test_accumulate_on_pipeline_sizes(B, dtype, M):
+    import torch
+    K, P = 7, 3 * 512 + 24
+    rng = np.random.default_rng(M)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    a = B.NbContext(K, P, M, 0.1, 0.9, "allreduce")
+    b = B.NbContext(K, P, M, 0.1, 0.9, "allreduce")
+    G = torch.from_numpy(rng.standard_normal((K, M, P)).astype(np.float32)).to(tdt).cuda()
+    n = rng.integers(0, M + 1, K)
+    n[0], n[1] = 0, M
+    flat = torch.empty(G.numel() + 1, dtype=tdt, device="cuda")
+    shifted = flat[1:].view_as(G)
+    shifted.copy_(G)
+    la = a.get_stats()["kernel_launches"]
+    a.accumulate(G, n)
+    assert a.get_stats()["kernel_launches"] - la == 2            # pipeline kernel + 24-column tail
+    b.accumulate(shifted, n)
+    acc = a.get_accumulator()
+    assert torch.equal(acc, b.get_accumulator())
+    H.assert_close(acc.numpy(), O.accumulate(G.float().cpu().numpy(), n.tolist()), 2e-6)
+    assert float(acc[0].abs().max()) == 0.0
+    a.close(); b.close()
