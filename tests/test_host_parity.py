@@ -148,3 +148,44 @@ def test_runtime_report_matches_oracle(name):
     with pytest.raises(B.NbError) as e:
         B.runtime_report("uniform_count", 1, 4, 4, 10)
     assert e.value.code == B.NB_ERR_UNSUPPORTED
+
+
+def test_randomised_straggler_configurations_bit_exact():
+    """Many random (model, K, M, means, seed, step) draws: counts, masks and times equal the oracle's."""
+    rng = np.random.default_rng(2211)
+    for _ in range(300):
+        K = int(rng.integers(1, 65))
+        M = int(rng.integers(1, 33))
+        seed = int(rng.integers(0, 2 ** 63))
+        t = int(rng.integers(0, 10 ** 9))
+        kind = int(rng.integers(0, 3))
+        if kind == 0:
+            model, params = "uniform_count", ()
+        elif kind == 1:
+            model, params = "shifted_exp", (float(rng.choice([0.0, 0.1, 0.5, 1.0, 2.0, 7.5])),)
+        else:
+            model, params = "shifted_exp_slowset", (float(rng.choice([0.0, 0.25, 0.5, 1.0])),
+                                                    float(rng.uniform(0, 4)), float(rng.uniform(0, 1)))
+        n, mask, tau = B.straggler_sample(model, seed, t, K, M, params)
+        want = O.straggler_counts(model, seed, t, K, M, params)
+        assert n.tolist() == want, (model, K, M, seed, t, params)
+        assert np.array_equal(mask, O.finished_mask(want, M))
+
+
+def test_randomised_regular_graphs_bit_exact():
+    rng = np.random.default_rng(889)
+    done = 0
+    while done < 16:
+        K = int(rng.integers(4, 41))
+        d = int(rng.integers(2, min(K - 1, 6) + 1))
+        if (K * d) % 2:
+            continue
+        seed = int(rng.integers(0, 2 ** 62))
+        topo, _ = B.make_topology("random_regular", degree=d, seed=seed, alpha=0.05, act_prob=0.5)
+        partner, attempts = B.topology_matchings(topo, K)
+        edges, want_attempts = O.random_regular_graph(seed, K, d)
+        assert attempts == want_attempts and partner.tolist() == O.greedy_matchings(edges, K)
+        for t in (0, 1, 12345):
+            _, bits = B.mixing_matrix(topo, B.NB_MATCHA, K, t)
+            assert bits == O.matcha_activation(seed, t, len(partner), 0.5)
+        done += 1
