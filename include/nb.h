@@ -82,8 +82,13 @@ typedef struct nb_topology {
   const float *val;        /* CSR: [row_ptr[K]]; rows and columns must sum to 1 within 1e-5        */
   int32_t n_matchings;     /* MATCHINGS: number of matchings, <= NB_MAX_MATCHINGS                  */
   const int32_t *partner;  /* MATCHINGS: [n_matchings*K], partner[c*K+v] = v's partner, -1 = none  */
-  float alpha;             /* MATCHA: W = I - alpha * sum_active L_j                               */
+  float alpha;             /* MATCHA: W = I - alpha * sum_active L_j, 0 <= alpha <= 1 (rows and     */
+                           /* columns always sum to 1; a diagonal entry is negative where alpha *   */
+                           /* active degree > 1)                                                    */
   float act_prob;          /* MATCHA: each matching is active with this probability, per step      */
+  const float *act_probs;  /* MATCHA: optional [number of matchings] per-matching probabilities    */
+                           /* (replace act_prob; for RANDOM_REGULAR learn the number of matchings  */
+                           /* from nb_topology_matchings first); NULL = act_prob for all           */
 } nb_topology;
 
 /* nb_set_option keys and values */
@@ -154,6 +159,19 @@ int nb_runtime_report_compute(const nb_straggler *cfg, int K, int M, int64_t ste
  * involution or repeats an edge; NB_ERR_UNSUPPORTED if more than NB_MAX_MATCHINGS are needed. */
 int nb_topology_matchings(const nb_topology *topo, int K, int32_t *partner, int32_t *n_matchings,
                           int32_t *attempts);
+
+/* MATCHA's design problem for the matchings of `topo` (MATCHINGS or RANDOM_REGULAR; Sec. 6.1: a
+ * communication budget c_b = mean activation frequency of the links, probabilities that favour the
+ * links that matter for connectivity, a step size alpha).  With L_bar(p) = sum_j p_j L_j:
+ *   probs  maximise lambda_2(L_bar(p)) subject to 0 <= p_j <= 1 and sum_j p_j <= budget * m
+ *          (projected supergradient ascent, `iters` iterations, 0 = 1000);
+ *   alpha  minimises rho = || E[W^T W] - (1/K) 1 1^T ||_2 for W = I - alpha * sum_j B_j L_j with
+ *          independent B_j ~ Bernoulli(p_j) (golden-section search on [0, 1]; rho is convex).
+ * Host out: probs[m] (m from nb_topology_matchings), *alpha, *lambda2, *rho (each may be NULL).
+ * budget = 1 gives p = 1: every matching always active, i.e. vanilla decentralized SGD.
+ * Errors: NB_ERR_ARG (bad topology, budget outside (0, 1]). */
+int nb_matcha_optimize(const nb_topology *topo, int K, float budget, int iters, float *probs, float *alpha,
+                       float *lambda2, float *rho);
 
 /* The mixing matrix a context created with (variant, topo, K) uses at `step`, dense row-major
  * host out [K*K]; bits: host out or NULL, the MATCHA activation word (bit j = matching j active).

@@ -298,6 +298,119 @@ def matcha_W(partner, bits, alpha, K):
 
 
 # ----------------------------------------------------------------------------------------------
+# MATCHA's design problem (Sec. 6.1 names it: a communication budget c_b = average activation
+# frequency of the links, probabilities that favour the links that matter for connectivity; the
+# optimisation itself is only referenced there, so it is stated here from first principles):
+#   L_bar(p) = sum_j p_j L_j                          expected Laplacian of the activated topology
+#   probabilities: maximise lambda_2(L_bar(p))  s.t.  0 <= p_j <= 1,  sum_j p_j <= c_b * m
+#   step size:     minimise rho(alpha) = || E[W^T W] - (1/K) 1 1^T ||_2,  W = I - alpha * L(k),
+#                  E[W^T W] = I - 2 alpha L_bar + alpha^2 (L_bar^2 + 2 sum_j p_j (1 - p_j) L_j)
+#                  (independent Bernoulli activations; L_j^2 = 2 L_j for a matching)
+# ----------------------------------------------------------------------------------------------
+def matching_laplacians(partner, K):
+    Ls = []
+    for row in partner:
+        L = np.zeros((K, K), dtype=np.float64)
+        for u in range(K):
+            v = row[u]
+            if v >= 0 and u < v:
+                L[u, u] += 1.0
+                L[v, v] += 1.0
+                L[u, v] -= 1.0
+                L[v, u] -= 1.0
+        Ls.append(L)
+    return Ls
+
+
+def matcha_lambda2(Ls, p):
+    """Algebraic connectivity (second smallest eigenvalue) of the expected Laplacian."""
+    Lbar = sum(float(pj) * L for pj, L in zip(p, Ls))
+    return float(np.linalg.eigvalsh(Lbar)[1])
+
+
+def project_budget(p, total):
+    """Euclidean projection onto {0 <= p_j <= 1, sum_j p_j <= total}."""
+    q = np.clip(p, 0.0, 1.0)
+    if q.sum() <= total:
+        return q
+    lo, hi = 0.0, float(np.max(p))
+    for _ in range(100):
+        mid = 0.5 * (lo + hi)
+        if np.clip(p - mid, 0.0, 1.0).sum() > total:
+            lo = mid
+        else:
+            hi = mid
+    return np.clip(p - hi, 0.0, 1.0)
+
+
+def matcha_optimal_probs(Ls, budget, iters=2000):
+    """Projected supergradient ascent on the concave function p -> lambda_2(L_bar(p)); a
+    supergradient is g_j = v^T L_j v for a unit Fiedler vector v.  Returns (p, lambda_2)."""
+    m = len(Ls)
+    total = float(budget) * m
+    p = project_budget(np.full(m, float(budget)), total)
+    best_p, best = p.copy(), matcha_lambda2(Ls, p)
+    for it in range(1, iters + 1):
+        Lbar = sum(pj * L for pj, L in zip(p, Ls))
+        w, V = np.linalg.eigh(Lbar)
+        v = V[:, 1]
+        g = np.array([float(v @ L @ v) for L in Ls])
+        nrm = float(np.linalg.norm(g))
+        if nrm == 0.0:
+            break
+        p = project_budget(p + (0.5 / math.sqrt(it)) * g / nrm, total)
+        val = matcha_lambda2(Ls, p)
+        if val > best:
+            best, best_p = val, p.copy()
+    return best_p, best
+
+
+def matcha_second_moment(Ls, p, alpha):
+    """E[W^T W] for W = I - alpha * sum_j B_j L_j with independent B_j ~ Bernoulli(p_j)."""
+    K = Ls[0].shape[0]
+    Lbar = sum(float(pj) * L for pj, L in zip(p, Ls))
+    Ltil = sum(float(pj) * (1.0 - float(pj)) * L for pj, L in zip(p, Ls))
+    return np.eye(K) - 2.0 * alpha * Lbar + alpha * alpha * (Lbar @ Lbar + 2.0 * Ltil)
+
+
+def matcha_rho(Ls, p, alpha):
+    """Spectral norm of E[W^T W] - J, J = (1/K) 1 1^T: the per-step contraction of the disagreement."""
+    K = Ls[0].shape[0]
+    A = matcha_second_moment(Ls, p, alpha) - np.full((K, K), 1.0 / K)
+    return float(np.max(np.abs(np.linalg.eigvalsh(A))))
+
+
+def matcha_optimal_alpha(Ls, p, iters=80):
+    """rho(alpha) is a maximum of convex quadratics in alpha, hence convex: golden-section search."""
+    lo, hi = 0.0, 1.0
+    gr = (math.sqrt(5.0) - 1.0) / 2.0
+    c, d = hi - gr * (hi - lo), lo + gr * (hi - lo)
+    fc, fd = matcha_rho(Ls, p, c), matcha_rho(Ls, p, d)
+    for _ in range(iters):
+        if fc < fd:
+            hi, d, fd = d, c, fc
+            c = hi - gr * (hi - lo)
+            fc = matcha_rho(Ls, p, c)
+        else:
+            lo, c, fc = c, d, fd
+            d = lo + gr * (hi - lo)
+            fd = matcha_rho(Ls, p, d)
+    a = 0.5 * (lo + hi)
+    return a, matcha_rho(Ls, p, a)
+
+
+def matcha_activation_probs(seed, t, probs):
+    """Activation word with one probability per matching (fp32 values widened, as the library
+    receives them): bit j = 1 iff the top 32 random bits fall below floor(p_j * 2^32)."""
+    bits = 0
+    for j, pj in enumerate(probs):
+        thr = int(math.floor(f32(pj) * 4294967296.0))
+        if (rng(seed, STREAM_MATCHA, t, j) >> 32) < thr:
+            bits |= (1 << j)
+    return bits
+
+
+# ----------------------------------------------------------------------------------------------
 # The step
 # ----------------------------------------------------------------------------------------------
 def accumulate(G, n):
@@ -410,7 +523,10 @@ class Oracle:
         if self.variant == "dpsgd":
             return self.W
         if self.variant == "matcha":
-            bits = matcha_activation(self.seed, t, len(self.partner), self.prob)
+            if isinstance(self.prob, (list, tuple, np.ndarray)):
+                bits = matcha_activation_probs(self.seed, t, self.prob)
+            else:
+                bits = matcha_activation(self.seed, t, len(self.partner), self.prob)
             return matcha_W(self.partner, bits, self.alpha, self.K)
         raise ValueError(self.variant)
 

@@ -33,7 +33,7 @@ class nb_topology(C.Structure):
     _fields_ = [("kind", C.c_int32), ("degree", C.c_int32), ("seed", C.c_uint64),
                 ("row_ptr", C.POINTER(C.c_int32)), ("col_idx", C.POINTER(C.c_int32)), ("val", C.POINTER(C.c_float)),
                 ("n_matchings", C.c_int32), ("partner", C.POINTER(C.c_int32)),
-                ("alpha", C.c_float), ("act_prob", C.c_float)]
+                ("alpha", C.c_float), ("act_prob", C.c_float), ("act_probs", C.POINTER(C.c_float))]
 
 
 class nb_runtime_report(C.Structure):
@@ -63,6 +63,7 @@ def _load():
     sig = {
         "nb_straggler_sample": [P(nb_straggler), i32, i32, i64, P(C.c_int32), P(C.c_uint8), P(C.c_double)],
         "nb_topology_matchings": [P(nb_topology), i32, P(C.c_int32), P(C.c_int32), P(C.c_int32)],
+        "nb_matcha_optimize": [P(nb_topology), i32, f32, i32, P(C.c_float), P(C.c_float), P(C.c_float), P(C.c_float)],
         "nb_mixing_matrix": [P(nb_topology), i32, i32, i64, P(C.c_float), P(C.c_uint32)],
         "nb_create": [P(vp), i32, i64, i32, f32, f32, i32, P(nb_topology)],
         "nb_destroy": [vp],
@@ -105,14 +106,15 @@ EXPORTED = ["nb_straggler_sample", "nb_topology_matchings", "nb_mixing_matrix", 
             "nb_step_fused", "nb_step_fused_host", "nb_get_params", "nb_get_momentum", "nb_get_accumulator",
             "nb_get_mean_params", "nb_set_state", "nb_get_step", "nb_get_W", "nb_get_matcha_activation",
             "nb_get_device_mixing", "nb_get_stats", "nb_step_static", "nb_get_kernel_plan",
-            "nb_begin_iteration", "nb_accumulate_minibatch", "nb_get_finished", "nb_runtime_report_compute"]
+            "nb_matcha_optimize", "nb_begin_iteration", "nb_accumulate_minibatch", "nb_get_finished", "nb_runtime_report_compute"]
 
 
 def _i32p(a):
     return a.ctypes.data_as(C.POINTER(C.c_int32))
 
 
-def make_topology(kind="full", K=0, degree=0, seed=0, csr=None, partner=None, alpha=0.0, act_prob=0.0):
+def make_topology(kind="full", K=0, degree=0, seed=0, csr=None, partner=None, alpha=0.0, act_prob=0.0,
+                  act_probs=None):
     """Returns (nb_topology, keepalive) for the named kind."""
     t = nb_topology()
     keep = []
@@ -130,6 +132,10 @@ def make_topology(kind="full", K=0, degree=0, seed=0, csr=None, partner=None, al
         keep += [rp, ci, va]
         t.row_ptr, t.col_idx = _i32p(rp), _i32p(ci)
         t.val = va.ctypes.data_as(C.POINTER(C.c_float))
+    if act_probs is not None:
+        ap = np.ascontiguousarray(act_probs, dtype=np.float32)
+        keep.append(ap)
+        t.act_probs = ap.ctypes.data_as(C.POINTER(C.c_float))
     if partner is not None:
         pt = np.ascontiguousarray(partner, dtype=np.int32)
         keep.append(pt)
@@ -177,6 +183,18 @@ def topology_matchings(topo, K):
     if rc != NB_OK:
         raise NbError(rc, "nb_topology_matchings")
     return partner[:n.value].copy(), att.value
+
+
+def matcha_optimize(topo, K, budget, iters=0):
+    """Activation probabilities (fp32 array [m]), alpha, lambda_2 and rho of MATCHA's design problem."""
+    m = topology_matchings(topo, K)[0].shape[0]
+    probs = np.zeros(m, dtype=np.float32)
+    a, l2, rho = C.c_float(0), C.c_float(0), C.c_float(0)
+    rc = lib.nb_matcha_optimize(C.byref(topo), K, budget, iters, probs.ctypes.data_as(C.POINTER(C.c_float)),
+                                C.byref(a), C.byref(l2), C.byref(rho))
+    if rc != NB_OK:
+        raise NbError(rc, "nb_matcha_optimize")
+    return probs, a.value, l2.value, rho.value
 
 
 def mixing_matrix(topo, variant, K, step):

@@ -160,7 +160,7 @@ int build_device_mixing(nb_ctx *c, cudaStream_t st) {
   m.mix = c->d_mix;
   m.partner = c->d_partner;
   m.seed = c->mx.seed;
-  m.thr = nb::activation_threshold(c->mx.act_prob);
+  for (int j = 0; j < c->mx.n_matchings; ++j) m.thr[j] = c->mx.thr[j];
   m.step = c->step;
   m.K = c->K;
   m.n_matchings = c->mx.n_matchings;
@@ -541,7 +541,7 @@ int nb_get_matcha_activation(nb_ctx *c, int64_t step, uint32_t *bits) {
   if (!c) return NB_ERR_ARG;
   if (!bits || step < 0) return fail(c, NB_ERR_ARG, "bits and step >= 0 required");
   if (c->variant != NB_MATCHA) return fail(c, NB_ERR_STATE, "not a MATCHA context");
-  *bits = nb::matcha_bits(c->mx.seed, step, c->mx.n_matchings, nb::activation_threshold(c->mx.act_prob));
+  *bits = nb::matcha_bits(c->mx.seed, step, c->mx.n_matchings, c->mx.thr.data());
   return NB_OK;
 }
 

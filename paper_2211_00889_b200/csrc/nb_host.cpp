@@ -192,17 +192,21 @@ int build_mixing(const nb_topology *topo, int variant, int K, Mixing *out, std::
       *err = "NB_MATCHA takes the MATCHINGS or RANDOM_REGULAR topology";
       return NB_ERR_ARG;
     }
-    if (!(topo->act_prob >= 0.f && topo->act_prob <= 1.f)) { *err = "act_prob must be in [0,1]"; return NB_ERR_ARG; }
-    // W must stay doubly stochastic with non-negative diagonal when every matching is active
-    std::vector<int> deg(K, 0);
-    for (int c = 0; c < mx.n_matchings; ++c)
-      for (int u = 0; u < K; ++u) deg[u] += mx.partner[(size_t)c * K + u] >= 0;
-    int dmax = 0;
-    for (int u = 0; u < K; ++u) dmax = std::max(dmax, deg[u]);
-    if (!(topo->alpha >= 0.f) || topo->alpha * (float)dmax > 1.0f) { *err = "alpha must satisfy 0 <= alpha*max_degree <= 1"; return NB_ERR_ARG; }
+    mx.probs.assign(mx.n_matchings, topo->act_prob);
+    if (topo->act_probs)
+      for (int c = 0; c < mx.n_matchings; ++c) mx.probs[c] = topo->act_probs[c];
+    else if (!(topo->act_prob >= 0.f && topo->act_prob <= 1.f)) { *err = "act_prob must be in [0,1]"; return NB_ERR_ARG; }
+    mx.thr.resize(mx.n_matchings);
+    for (int c = 0; c < mx.n_matchings; ++c) {
+      if (!(mx.probs[c] >= 0.f && mx.probs[c] <= 1.f)) { *err = "activation probabilities must be in [0,1]"; return NB_ERR_ARG; }
+      mx.thr[c] = activation_threshold(mx.probs[c]);
+    }
+    // rows and columns of W = I - alpha * sum_active L_j sum to one for every alpha; alpha <= 1 keeps
+    // every I - alpha * L_j a contraction (a vertex whose active degree exceeds 1/alpha gets a
+    // negative diagonal weight, which MATCHA's optimal step sizes do produce)
+    if (!(topo->alpha >= 0.f && topo->alpha <= 1.0f)) { *err = "alpha must be in [0, 1]"; return NB_ERR_ARG; }
     if ((size_t)K * (size_t)(1 + mx.n_matchings) > NB_MAX_NNZ) { *err = "K*(1+matchings) exceeds NB_MAX_NNZ"; return NB_ERR_UNSUPPORTED; }
     mx.alpha = topo->alpha;
-    mx.act_prob = topo->act_prob;
     mx.seed = topo->seed;
     *out = mx;
     return NB_OK;
@@ -221,7 +225,7 @@ void dense_W(const Mixing &mx, int64_t step, float *W, uint32_t *bits) {
     for (int i = 0; i < K; ++i)
       for (int e = mx.row_ptr[i]; e < mx.row_ptr[i + 1]; ++e) W[(size_t)i * K + mx.col[e]] = mx.val[e];
   } else {
-    b = matcha_bits(mx.seed, step, mx.n_matchings, activation_threshold(mx.act_prob));
+    b = matcha_bits(mx.seed, step, mx.n_matchings, mx.thr.data());
     for (int i = 0; i < K; ++i) {
       int cnt = 0;
       for (int c = 0; c < mx.n_matchings; ++c) {
@@ -235,6 +239,181 @@ void dense_W(const Mixing &mx, int64_t step, float *W, uint32_t *bits) {
 }
 
 }  // namespace nb
+
+namespace nb {
+namespace {
+
+// Cyclic Jacobi eigenvalue iteration for a symmetric n x n matrix (row-major, destroyed).
+// Eigenvalues ascending in w, matching unit eigenvectors in the columns of V.
+void jacobi_eigh(std::vector<double> &A, int n, std::vector<double> &w, std::vector<double> &V) {
+  V.assign((size_t)n * n, 0.0);
+  for (int i = 0; i < n; ++i) V[(size_t)i * n + i] = 1.0;
+  for (int sweep = 0; sweep < 60; ++sweep) {
+    double off = 0.0;
+    for (int p = 0; p < n; ++p)
+      for (int q = p + 1; q < n; ++q) off += A[(size_t)p * n + q] * A[(size_t)p * n + q];
+    if (off < 1e-26) break;
+    for (int p = 0; p < n; ++p)
+      for (int q = p + 1; q < n; ++q) {
+        const double apq = A[(size_t)p * n + q];
+        if (std::fabs(apq) < 1e-300) continue;
+        const double theta = (A[(size_t)q * n + q] - A[(size_t)p * n + p]) / (2.0 * apq);
+        const double t = (theta >= 0 ? 1.0 : -1.0) / (std::fabs(theta) + std::sqrt(theta * theta + 1.0));
+        const double c = 1.0 / std::sqrt(t * t + 1.0), sn = t * c;
+        for (int k = 0; k < n; ++k) {  // columns p, q
+          const double akp = A[(size_t)k * n + p], akq = A[(size_t)k * n + q];
+          A[(size_t)k * n + p] = c * akp - sn * akq;
+          A[(size_t)k * n + q] = sn * akp + c * akq;
+        }
+        for (int k = 0; k < n; ++k) {  // rows p, q
+          const double apk = A[(size_t)p * n + k], aqk = A[(size_t)q * n + k];
+          A[(size_t)p * n + k] = c * apk - sn * aqk;
+          A[(size_t)q * n + k] = sn * apk + c * aqk;
+        }
+        for (int k = 0; k < n; ++k) {
+          const double vkp = V[(size_t)k * n + p], vkq = V[(size_t)k * n + q];
+          V[(size_t)k * n + p] = c * vkp - sn * vkq;
+          V[(size_t)k * n + q] = sn * vkp + c * vkq;
+        }
+      }
+  }
+  std::vector<int> idx(n);
+  for (int i = 0; i < n; ++i) idx[i] = i;
+  std::sort(idx.begin(), idx.end(), [&](int a, int b) { return A[(size_t)a * n + a] < A[(size_t)b * n + b]; });
+  w.resize(n);
+  std::vector<double> Vs((size_t)n * n);
+  for (int j = 0; j < n; ++j) {
+    w[j] = A[(size_t)idx[j] * n + idx[j]];
+    for (int k = 0; k < n; ++k) Vs[(size_t)k * n + j] = V[(size_t)k * n + idx[j]];
+  }
+  V.swap(Vs);
+}
+
+// sum_j p_j L_j for the matchings in `partner`
+void expected_laplacian(const std::vector<int32_t> &partner, int m, int K, const std::vector<double> &p,
+                        std::vector<double> &L) {
+  L.assign((size_t)K * K, 0.0);
+  for (int c = 0; c < m; ++c)
+    for (int u = 0; u < K; ++u) {
+      const int v = partner[(size_t)c * K + u];
+      if (v > u) {
+        L[(size_t)u * K + u] += p[c];
+        L[(size_t)v * K + v] += p[c];
+        L[(size_t)u * K + v] -= p[c];
+        L[(size_t)v * K + u] -= p[c];
+      }
+    }
+}
+
+// Euclidean projection onto {0 <= p_j <= 1, sum p_j <= total}
+void project_budget(std::vector<double> &p, double total) {
+  std::vector<double> raw = p;
+  double sum = 0.0, pmax = 0.0;
+  for (auto &x : p) { x = std::min(1.0, std::max(0.0, x)); sum += x; }
+  if (sum <= total) return;
+  for (double x : raw) pmax = std::max(pmax, x);
+  double lo = 0.0, hi = pmax;
+  for (int it = 0; it < 100; ++it) {
+    const double mid = 0.5 * (lo + hi);
+    double sm = 0.0;
+    for (double x : raw) sm += std::min(1.0, std::max(0.0, x - mid));
+    if (sm > total) lo = mid; else hi = mid;
+  }
+  for (size_t j = 0; j < p.size(); ++j) p[j] = std::min(1.0, std::max(0.0, raw[j] - hi));
+}
+
+double lambda2_of(const std::vector<int32_t> &partner, int m, int K, const std::vector<double> &p,
+                  std::vector<double> *fiedler) {
+  std::vector<double> L, w, V;
+  expected_laplacian(partner, m, K, p, L);
+  jacobi_eigh(L, K, w, V);
+  if (K < 2) return 0.0;
+  if (fiedler) {
+    fiedler->resize(K);
+    for (int k = 0; k < K; ++k) (*fiedler)[k] = V[(size_t)k * K + 1];
+  }
+  return w[1];
+}
+
+// || E[W^T W] - J ||_2 with E[W^T W] = I - 2a L_bar + a^2 (L_bar^2 + 2 sum_j p_j (1 - p_j) L_j)
+double rho_of(const std::vector<int32_t> &partner, int m, int K, const std::vector<double> &p, double a) {
+  std::vector<double> Lb, Lt, pt(m);
+  for (int c = 0; c < m; ++c) pt[c] = p[c] * (1.0 - p[c]);
+  expected_laplacian(partner, m, K, p, Lb);
+  expected_laplacian(partner, m, K, pt, Lt);
+  std::vector<double> A((size_t)K * K);
+  for (int i = 0; i < K; ++i)
+    for (int j = 0; j < K; ++j) {
+      double l2 = 0.0;
+      for (int k = 0; k < K; ++k) l2 += Lb[(size_t)i * K + k] * Lb[(size_t)k * K + j];
+      A[(size_t)i * K + j] = (i == j ? 1.0 : 0.0) - 2.0 * a * Lb[(size_t)i * K + j] +
+                             a * a * (l2 + 2.0 * Lt[(size_t)i * K + j]) - 1.0 / (double)K;
+    }
+  std::vector<double> w, V;
+  jacobi_eigh(A, K, w, V);
+  return std::max(std::fabs(w[0]), std::fabs(w[K - 1]));
+}
+
+}  // namespace
+}  // namespace nb
+
+extern "C" int nb_matcha_optimize(const nb_topology *topo, int K, float budget, int iters, float *probs, float *alpha,
+                                  float *lambda2, float *rho) {
+  using namespace nb;
+  if (!topo || !(budget > 0.f && budget <= 1.f) || iters < 0) return NB_ERR_ARG;
+  Mixing mx;
+  std::string err;
+  nb_topology t = *topo;
+  t.alpha = 0.f;
+  t.act_prob = 0.f;
+  t.act_probs = nullptr;
+  int st = build_mixing(&t, NB_MATCHA, K, &mx, &err);
+  if (st != NB_OK) return st;
+  const int m = mx.n_matchings;
+  if (m < 1 || K < 2) return NB_ERR_ARG;
+  if (iters == 0) iters = 1000;
+  const double total = (double)budget * m;
+  std::vector<double> p(m, (double)budget), best_p, fied, g(m);
+  project_budget(p, total);
+  best_p = p;
+  double best = lambda2_of(mx.partner, m, K, p, &fied);
+  for (int it = 1; it <= iters; ++it) {
+    double nrm = 0.0;
+    for (int c = 0; c < m; ++c) {  // supergradient g_c = v^T L_c v = sum over the matching's edges of (v_u - v_w)^2
+      double s = 0.0;
+      for (int u = 0; u < K; ++u) {
+        const int v = mx.partner[(size_t)c * K + u];
+        if (v > u) s += (fied[u] - fied[v]) * (fied[u] - fied[v]);
+      }
+      g[c] = s;
+      nrm += s * s;
+    }
+    nrm = std::sqrt(nrm);
+    if (nrm == 0.0) break;
+    const double step = 0.5 / std::sqrt((double)it);
+    for (int c = 0; c < m; ++c) p[c] += step * g[c] / nrm;
+    project_budget(p, total);
+    const double val = lambda2_of(mx.partner, m, K, p, &fied);
+    if (val > best) { best = val; best_p = p; }
+  }
+  // the library consumes fp32 probabilities: evaluate alpha and rho at the rounded values
+  std::vector<double> pf(m);
+  for (int c = 0; c < m; ++c) pf[c] = (double)(float)best_p[c];
+  double lo = 0.0, hi = 1.0;
+  const double gr = (std::sqrt(5.0) - 1.0) / 2.0;
+  double c1 = hi - gr * (hi - lo), d1 = lo + gr * (hi - lo);
+  double fc = rho_of(mx.partner, m, K, pf, c1), fd = rho_of(mx.partner, m, K, pf, d1);
+  for (int it = 0; it < 80; ++it) {
+    if (fc < fd) { hi = d1; d1 = c1; fd = fc; c1 = hi - gr * (hi - lo); fc = rho_of(mx.partner, m, K, pf, c1); }
+    else { lo = c1; c1 = d1; fc = fd; d1 = lo + gr * (hi - lo); fd = rho_of(mx.partner, m, K, pf, d1); }
+  }
+  const float a = (float)(0.5 * (lo + hi));
+  if (probs) for (int c = 0; c < m; ++c) probs[c] = (float)best_p[c];
+  if (alpha) *alpha = a;
+  if (lambda2) *lambda2 = (float)lambda2_of(mx.partner, m, K, pf, nullptr);
+  if (rho) *rho = (float)rho_of(mx.partner, m, K, pf, (double)a);
+  return NB_OK;
+}
 
 // -------------------------------------------------------------------------------------------------
 // C ABI: host-only entry points
@@ -296,9 +475,10 @@ extern "C" int nb_topology_matchings(const nb_topology *topo, int K, int32_t *pa
   std::string err;
   nb_topology t = *topo;
   if (t.kind == NB_TOPO_RANDOM_REGULAR || t.kind == NB_TOPO_MATCHINGS) {
-    // alpha / act_prob do not matter for the decomposition itself
+    // alpha / activation probabilities do not matter for the decomposition itself
     t.alpha = 0.f;
     t.act_prob = 0.f;
+    t.act_probs = nullptr;
   }
   int st = nb::build_mixing(&t, NB_MATCHA, K, &mx, &err);
   if (st != NB_OK) return st;

@@ -39,10 +39,11 @@ NB_HD uint64_t activation_threshold(float prob) {
   if (t >= 4294967296.0) return 4294967296ull;
   return (uint64_t)t;
 }
-NB_HD uint32_t matcha_bits(uint64_t seed, int64_t step, int n_matchings, uint64_t thr) {
+// One independent Bernoulli draw per matching per step; thr[j] = activation_threshold(p_j).
+NB_HD uint32_t matcha_bits(uint64_t seed, int64_t step, int n_matchings, const uint64_t *thr) {
   uint32_t bits = 0;
   for (int j = 0; j < n_matchings; ++j)
-    if ((rng(seed, kMatcha, (uint64_t)step, (uint64_t)j) >> 32) < thr) bits |= (1u << j);
+    if ((rng(seed, kMatcha, (uint64_t)step, (uint64_t)j) >> 32) < thr[j]) bits |= (1u << j);
   return bits;
 }
 
@@ -58,7 +59,9 @@ struct Mixing {
   // NB_MATCHA
   int n_matchings = 0;
   std::vector<int32_t> partner;  // [n_matchings*K]
-  float alpha = 0.f, act_prob = 0.f;
+  float alpha = 0.f;
+  std::vector<float> probs;      // [n_matchings] activation probabilities
+  std::vector<uint64_t> thr;     // [n_matchings] activation thresholds
   uint64_t seed = 0;
   int attempts = 0;
 };

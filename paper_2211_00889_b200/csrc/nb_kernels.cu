@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(256) nb_centralized_kernel(const __grid_consta
 // K3: MATCHA activation + W builder.  One Bernoulli draw per matching per step from the counter
 // generator; row i of W = I - alpha * sum_active L_j is written as (diagonal, active partners).
 // -------------------------------------------------------------------------------------------------
-__global__ void nb_matcha_build_kernel(const MatchaArgs a) {
+__global__ void nb_matcha_build_kernel(const __grid_constant__ MatchaArgs a) {
   const int i = threadIdx.x;
   const uint32_t bits = matcha_bits(a.seed, a.step, a.n_matchings, a.thr);
   const int stride = 1 + a.n_matchings;

@@ -43,7 +43,8 @@ struct StepArgs {
 struct MatchaArgs {
   MixTable *mix;
   const int32_t *partner;  // device [n_matchings*K]
-  uint64_t seed, thr;
+  uint64_t seed;
+  uint64_t thr[NB_MAX_MATCHINGS];  // per-matching activation thresholds
   int64_t step;
   int32_t K, n_matchings;
   float alpha;

@@ -417,3 +417,35 @@ def test_streaming_accumulate_follows_alg1_and_equals_batch_accumulate(B):
         assert torch.equal(a.get_params(), b.get_params())
     H.assert_close(a.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
     a.close(); b.close()
+
+
+def test_matcha_with_optimised_per_matching_probabilities(B):
+    """MATCHA's designed topology: per-matching activation probabilities under a budget and the
+    optimal alpha from nb_matcha_optimize; activation words bit-exact on device, host and oracle."""
+    import torch
+    K, P, M = 16, 3 * 512 + 40, 4
+    seed = 221100893
+    base, _ = B.make_topology("random_regular", degree=3, seed=seed)
+    probs, alpha, lam2, rho = B.matcha_optimize(base, K, 0.5)
+    assert 0 < rho < 1 and lam2 > 0
+    partner, _ = B.topology_matchings(base, K)
+    topo = B.make_topology("random_regular", degree=3, seed=seed, alpha=alpha, act_probs=probs)
+    ctx = B.NbContext(K, P, M, 0.05, 0.9, "matcha", topo)
+    orc = O.Oracle(K, P, M, 0.05, 0.9, "matcha", partner=partner.tolist(), alpha=alpha, prob=probs.tolist(), seed=seed)
+    rng = np.random.default_rng(1)
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    ctx.set_params(torch.from_numpy(x0).cuda()); orc.set_params(x0)
+    seen = set()
+    for t in range(8):
+        G = torch.from_numpy((rng.standard_normal((K, M, P)) * 0.01).astype(np.float32)).to(torch.bfloat16).cuda()
+        n = rng.integers(1, M + 1, K)
+        ctx.step_fused(G, n)
+        orc.step(G.float().cpu().numpy(), n.tolist())
+        bits, Wdev = ctx.get_device_mixing()
+        assert bits == O.matcha_activation_probs(seed, t, probs.tolist()) == ctx.get_matcha_activation(t)
+        assert np.array_equal(Wdev, ctx.get_W(t))
+        assert np.allclose(Wdev.sum(0), 1.0, atol=1e-6) and np.allclose(Wdev.sum(1), 1.0, atol=1e-6)
+        seen.add(bits)
+    assert len(seen) > 1
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+    ctx.close()

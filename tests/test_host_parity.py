@@ -117,8 +117,8 @@ def test_topology_validation():
     # edge repeated in two matchings
     topo, keep = B.make_topology("matchings", partner=np.array([[1, 0, -1, -1], [1, 0, 3, 2]]), alpha=0.1, act_prob=0.5)
     assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_MATCHA, 4, 0, Wp, None) == B.NB_ERR_ARG
-    # alpha too large for the degree
-    topo, keep = B.make_topology("matchings", partner=np.array([[1, 0, 3, 2], [2, 3, 0, 1]]), alpha=0.6, act_prob=0.5)
+    # alpha outside [0, 1]
+    topo, keep = B.make_topology("matchings", partner=np.array([[1, 0, 3, 2], [2, 3, 0, 1]]), alpha=1.5, act_prob=0.5)
     assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_MATCHA, 4, 0, Wp, None) == B.NB_ERR_ARG
     # impossible regular graph (odd K*d)
     topo, keep = B.make_topology("random_regular", degree=3, seed=1, alpha=0.1, act_prob=0.5)
@@ -189,3 +189,49 @@ def test_randomised_regular_graphs_bit_exact():
             _, bits = B.mixing_matrix(topo, B.NB_MATCHA, K, t)
             assert bits == O.matcha_activation(seed, t, len(partner), 0.5)
         done += 1
+
+
+@pytest.mark.parametrize("seed,K,d,budget", [(221100893, 16, 3, 0.5), (7, 12, 3, 0.3), (11, 20, 4, 0.6), (3, 8, 3, 1.0)])
+def test_matcha_design_problem_matches_oracle_optimum(seed, K, d, budget):
+    """Activation probabilities and alpha from the library solve the same two problems as the
+    oracle's routines: compared through the optimal VALUES (the maximiser need not be unique)."""
+    topo, _ = B.make_topology("random_regular", degree=d, seed=seed)
+    probs, alpha, lam2, rho = B.matcha_optimize(topo, K, budget, iters=1500)
+    partner, _ = B.topology_matchings(topo, K)
+    m = len(partner)
+    Ls = O.matching_laplacians(partner.tolist(), K)
+    assert probs.shape == (m,) and np.all(probs >= 0) and np.all(probs <= 1)
+    assert probs.sum() <= budget * m + 1e-4                                   # the budget holds
+    p_or, lam_or = O.matcha_optimal_probs(Ls, budget, iters=1500)
+    assert O.matcha_lambda2(Ls, probs) == pytest.approx(lam2, rel=1e-4, abs=1e-6)
+    assert lam2 == pytest.approx(lam_or, rel=2e-3, abs=1e-5)                   # same optimum
+    assert lam2 >= O.matcha_lambda2(Ls, [budget] * m) - 1e-6                   # never worse than uniform spending
+    a_or, rho_or = O.matcha_optimal_alpha(Ls, probs)                           # oracle's alpha for the library's p
+    assert O.matcha_rho(Ls, probs, alpha) == pytest.approx(rho, rel=1e-4)
+    assert rho == pytest.approx(rho_or, rel=1e-4) and abs(alpha - a_or) < 2e-3
+    assert 0.0 < rho < 1.0
+    if budget == 1.0:
+        assert np.allclose(probs, 1.0)
+
+
+def test_per_matching_probabilities_drive_the_activation_words():
+    K = 16
+    topo, _ = B.make_topology("random_regular", degree=3, seed=221100893)
+    probs, alpha, _, _ = B.matcha_optimize(topo, K, 0.5)
+    partner, _ = B.topology_matchings(topo, K)
+    topo2, keep = B.make_topology("random_regular", degree=3, seed=221100893, alpha=alpha, act_probs=probs)
+    freq = np.zeros(len(partner))
+    T = 3000
+    for t in range(T):
+        W, bits = B.mixing_matrix(topo2, B.NB_MATCHA, K, t)
+        assert bits == O.matcha_activation_probs(221100893, t, probs.tolist())   # bit-exact
+        Wd = O.matcha_W(partner.tolist(), bits, alpha, K)
+        assert np.abs(W.astype(np.float64) - Wd).max() < 1e-6
+        for j in range(len(partner)):
+            freq[j] += (bits >> j) & 1
+    assert np.all(np.abs(freq / T - probs) < 0.04)
+    # a probability outside [0, 1] is rejected
+    import ctypes as C
+    bad, keep2 = B.make_topology("random_regular", degree=3, seed=1, alpha=0.1, act_probs=np.array([0.5, 1.5, 0.5, 0.5, 0.5]))
+    Wbuf = np.zeros((K, K), dtype=np.float32)
+    assert B.lib.nb_mixing_matrix(C.byref(bad), B.NB_MATCHA, K, 0, Wbuf.ctypes.data_as(C.POINTER(C.c_float)), None) == B.NB_ERR_ARG

@@ -521,3 +521,90 @@ def test_centralized_step_equals_synchronous_sgd_and_the_allreduce_mean():
 def test_mean_params():
     X = np.arange(12.0).reshape(3, 4)
     assert O.mean_params(X).tolist() == [4.0, 5.0, 6.0, 7.0]
+
+
+# ------------------------------------------------------------------------------------------
+# MATCHA's design problem: activation probabilities under a budget, step size alpha
+# ------------------------------------------------------------------------------------------
+def _path_matchings():
+    # path 0-1-2-3-4-5 split into two matchings; plus a chord matching {0-5}
+    return [[1, 0, 3, 2, 5, 4], [-1, 2, 1, 4, 3, -1], [5, -1, -1, -1, -1, 0]]
+
+
+def test_second_moment_closed_form_equals_enumeration_over_activation_patterns():
+    K = 6
+    partner = _path_matchings()
+    Ls = O.matching_laplacians(partner, K)
+    p, alpha = [0.7, 0.35, 0.9], 0.3
+    want = np.zeros((K, K))
+    for pattern in range(8):                                   # all 2^m activation patterns, exactly
+        prob = 1.0
+        for j in range(3):
+            prob *= p[j] if (pattern >> j) & 1 else 1.0 - p[j]
+        W = np.eye(K) - alpha * sum((Ls[j] for j in range(3) if (pattern >> j) & 1), np.zeros((K, K)))
+        want += prob * (W.T @ W)
+    assert np.allclose(O.matcha_second_moment(Ls, p, alpha), want, rtol=0, atol=1e-14)
+    for L in Ls:                                                 # the identity the closed form rests on
+        assert np.array_equal(L @ L, 2.0 * L)
+
+
+def test_probability_projection():
+    q = O.project_budget(np.array([0.9, 0.8, -0.2, 1.4]), 10.0)
+    assert q.tolist() == [0.9, 0.8, 0.0, 1.0]
+    q = O.project_budget(np.array([0.9, 0.8, 0.7]), 1.2)
+    assert abs(q.sum() - 1.2) < 1e-9 and np.all(q >= 0) and np.all(q <= 1)
+    assert np.allclose(q - q[0], np.array([0.0, -0.1, -0.2]), atol=1e-9)   # equal shift of the free coordinates
+    # brute force: no feasible grid point is closer
+    target = np.array([0.9, 0.8, 0.7])
+    best = min(((np.array([a, b, c]) - target) @ (np.array([a, b, c]) - target))
+               for a in np.linspace(0, 1, 41) for b in np.linspace(0, 1, 41) for c in np.linspace(0, 1, 41)
+               if a + b + c <= 1.2 + 1e-12)
+    assert (q - target) @ (q - target) <= best + 1e-9
+
+
+def test_optimal_probabilities_against_grid_search():
+    K = 6
+    Ls = O.matching_laplacians(_path_matchings(), K)
+    budget = 0.5
+    p, lam = O.matcha_optimal_probs(Ls, budget, iters=1500)
+    assert np.all(p >= -1e-12) and np.all(p <= 1 + 1e-12) and p.sum() <= budget * 3 + 1e-9
+    grid = np.linspace(0, 1, 51)
+    best = max(O.matcha_lambda2(Ls, (a, b, c)) for a in grid for b in grid for c in grid
+               if a + b + c <= budget * 3 + 1e-12)
+    assert lam >= best - 1e-4                                    # as good as any grid point (iteration accuracy)
+    assert lam <= best + 0.02                                    # and the grid (step 0.02) nearly reaches it
+    assert lam > O.matcha_lambda2(Ls, [budget] * 3) + 1e-3       # better than spending the budget uniformly
+    # full budget: every matching always active
+    p1, lam1 = O.matcha_optimal_probs(Ls, 1.0, iters=200)
+    assert np.allclose(p1, 1.0) and lam1 == pytest.approx(O.matcha_lambda2(Ls, [1, 1, 1]))
+
+
+def test_optimal_alpha_against_grid_and_contraction():
+    K = 16
+    edges, _ = O.random_regular_graph(221100893, K, 3)
+    partner = O.greedy_matchings(edges, K)
+    Ls = O.matching_laplacians(partner, K)
+    p, lam = O.matcha_optimal_probs(Ls, 0.5, iters=800)
+    assert lam > 0                                               # expected topology is connected
+    a, rho = O.matcha_optimal_alpha(Ls, p)
+    grid = np.linspace(0.0, 1.0, 2001)
+    vals = [O.matcha_rho(Ls, p, x) for x in grid]
+    assert rho <= min(vals) + 1e-9 and abs(a - grid[int(np.argmin(vals))]) < 2e-3
+    assert 0.0 < rho < 1.0                                       # mixing contracts the disagreement
+    assert O.matcha_rho(Ls, p, 0.0) == pytest.approx(1.0)        # alpha = 0: W = I, no mixing
+    # rho is convex in alpha
+    assert all(vals[i] <= 0.5 * (vals[i - 1] + vals[i + 1]) + 1e-12 for i in range(1, len(vals) - 1))
+
+
+def test_activation_with_per_matching_probabilities():
+    probs = [0.0, 1.0, 0.25, 0.75]
+    freq = np.zeros(4)
+    T = 8000
+    for t in range(T):
+        bits = O.matcha_activation_probs(5, t, probs)
+        for j in range(4):
+            freq[j] += (bits >> j) & 1
+    assert freq[0] == 0 and freq[1] == T
+    assert abs(freq[2] / T - 0.25) < 0.02 and abs(freq[3] / T - 0.75) < 0.02
+    # equal probabilities reduce to the single-probability form
+    assert all(O.matcha_activation_probs(9, t, [0.5] * 5) == O.matcha_activation(9, t, 5, 0.5) for t in range(200))
