@@ -35,7 +35,7 @@ DEFAULT_WORKLOAD = "cfg3_dpsgd_ring_resnet50"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per algorithmic byte of the fused step kernel: dram__bytes_read.sum + dram__bytes_write.sum
 # of nb_step_pipeline_kernel over the algorithmic bytes of the same launch, from the ncu capture of an
-# 8M-column case of the default workload (profiles/nb_step_pipeline_kernel_cfg3_8Mcols_traffic.md).
+# 8M-column case of the default workload (summarised under profiles/).
 # Traffic grows in proportion to the columns a launch processes.
 TRAFFIC_PER_ALGORITHMIC_BYTE = 0.988
 
