@@ -273,6 +273,12 @@ int nb_get_device_mixing(nb_ctx *c, uint32_t *bits, float *W_dense, void *stream
 int nb_get_stats(const nb_ctx *c, int64_t *sum_finished, double *algorithmic_bytes,
                  int64_t *kernel_launches);
 
+/* Self-check: X, V and the accumulator are allocated between guard bands of a fixed byte pattern;
+ * this waits for `stream`, reads the bands back and returns NB_ERR_STATE (with the array and offset
+ * in nb_last_error) if any kernel wrote outside its array, NB_ERR_CUDA if a kernel reported a wait
+ * that ran out, NB_OK otherwise. */
+int nb_check_guards(nb_ctx *c, void *stream);
+
 /* Which kernel shape ran the most recent step (for reports and tests), host out plan[8]:
  * [0] 1 if the bulk-copy pipeline kernel covered the full tiles, 0 if the direct-load kernel did
  * everything; [1] tile width in columns; [2] consumer groups per CTA; [3] ring slots per CTA;

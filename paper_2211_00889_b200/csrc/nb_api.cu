@@ -18,6 +18,10 @@ struct nb_ctx {
   int variant = NB_ALLREDUCE, norm = NB_NORM_MEAN, order = NB_ORDER_MIX_THEN_UPDATE;
   nb::Mixing mx;
   float *X = nullptr, *V = nullptr, *acc = nullptr, *d_mean = nullptr;
+  // X, V and acc sit between guard bands (kGuardBytes of a fixed byte pattern before and after);
+  // nb_check_guards verifies that no kernel wrote outside its arrays.
+  unsigned char *X_base = nullptr, *V_base = nullptr, *acc_base = nullptr;
+  size_t model_bytes = 0, acc_bytes = 0;
   nb::MixTable *d_mix = nullptr;
   int32_t *d_partner = nullptr;
   int *d_err = nullptr;  // device word a kernel sets when one of its bounded waits runs out
@@ -38,6 +42,20 @@ struct nb_ctx {
 namespace {
 
 thread_local std::string g_create_err;
+
+constexpr size_t kGuardBytes = 1024;
+constexpr int kGuardPattern = 0xA5;
+
+// One array with a guard band on each side; *data is 1024-byte aligned.
+cudaError_t alloc_guarded(unsigned char **base, float **data, size_t bytes) {
+  cudaError_t e = cudaMalloc(base, bytes + 2 * kGuardBytes);
+  if (e != cudaSuccess) return e;
+  if ((e = cudaMemset(*base, kGuardPattern, kGuardBytes)) != cudaSuccess) return e;
+  if ((e = cudaMemset(*base + kGuardBytes, 0, bytes)) != cudaSuccess) return e;
+  if ((e = cudaMemset(*base + kGuardBytes + bytes, kGuardPattern, kGuardBytes)) != cudaSuccess) return e;
+  *data = reinterpret_cast<float *>(*base + kGuardBytes);
+  return cudaSuccess;
+}
 
 struct DeviceGuard {
   int prev = -1;
@@ -259,12 +277,11 @@ int nb_create(nb_ctx **out, int K, int64_t P, int M, float lr, float mom, int va
   if ((e = nb::configure_kernels()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute");
   const size_t model_bytes = sizeof(float) * (size_t)c->rows * (size_t)c->ldx;
   const size_t acc_bytes = sizeof(float) * (size_t)K * (size_t)c->ldx;
-  if ((e = cudaMalloc(&c->X, model_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(X)");
-  if ((e = cudaMalloc(&c->V, model_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(V)");
-  if ((e = cudaMalloc(&c->acc, acc_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(acc)");
-  if ((e = cudaMemset(c->X, 0, model_bytes)) != cudaSuccess) return bail(e, "cudaMemset(X)");
-  if ((e = cudaMemset(c->V, 0, model_bytes)) != cudaSuccess) return bail(e, "cudaMemset(V)");
-  if ((e = cudaMemset(c->acc, 0, acc_bytes)) != cudaSuccess) return bail(e, "cudaMemset(acc)");
+  c->model_bytes = model_bytes;
+  c->acc_bytes = acc_bytes;
+  if ((e = alloc_guarded(&c->X_base, &c->X, model_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(X)");
+  if ((e = alloc_guarded(&c->V_base, &c->V, model_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(V)");
+  if ((e = alloc_guarded(&c->acc_base, &c->acc, acc_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(acc)");
   if ((e = cudaMalloc(&c->d_err, sizeof(int))) != cudaSuccess) return bail(e, "cudaMalloc(err)");
   if ((e = cudaMemset(c->d_err, 0, sizeof(int))) != cudaSuccess) return bail(e, "cudaMemset(err)");
   if (variant == NB_DPSGD || variant == NB_MATCHA) {
@@ -295,9 +312,9 @@ int nb_destroy(nb_ctx *c) {
   if (!c) return NB_OK;
   DeviceGuard guard(c->device);
   cudaDeviceSynchronize();
-  cudaFree(c->X);
-  cudaFree(c->V);
-  cudaFree(c->acc);
+  cudaFree(c->X_base);
+  cudaFree(c->V_base);
+  cudaFree(c->acc_base);
   cudaFree(c->d_mean);
   cudaFree(c->d_mix);
   cudaFree(c->d_partner);
@@ -567,6 +584,26 @@ int nb_get_device_mixing(nb_ctx *c, uint32_t *bits, float *W_dense, void *stream
   }
   delete h;
   return NB_OK;
+}
+
+int nb_check_guards(nb_ctx *c, void *stream) {
+  NB_ENTER(c);
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned char h[2 * kGuardBytes];
+  struct Arr { const char *name; unsigned char *base; size_t bytes; };
+  const Arr arrs[3] = {{"X", c->X_base, c->model_bytes}, {"V", c->V_base, c->model_bytes}, {"acc", c->acc_base, c->acc_bytes}};
+  for (const Arr &a : arrs) {
+    NB_CUDA(c, cudaMemcpyAsync(h, a.base, kGuardBytes, cudaMemcpyDeviceToHost, st));
+    NB_CUDA(c, cudaMemcpyAsync(h + kGuardBytes, a.base + kGuardBytes + a.bytes, kGuardBytes, cudaMemcpyDeviceToHost, st));
+    NB_CUDA(c, cudaStreamSynchronize(st));
+    for (size_t q = 0; q < 2 * kGuardBytes; ++q)
+      if (h[q] != kGuardPattern)
+        return fail(c, NB_ERR_STATE, std::string("guard band of ") + a.name + " overwritten at byte " +
+                                         std::to_string(q < kGuardBytes ? (long long)q - (long long)kGuardBytes
+                                                                        : (long long)(q - kGuardBytes)) +
+                                         (q < kGuardBytes ? " before the array" : " after the array"));
+  }
+  return check_device_error(c, st);
 }
 
 int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan) {

@@ -68,6 +68,7 @@ def test_full_size_sampled_columns(name, steps):
     torch.cuda.empty_cache()
     X = ctx.get_params(device="cuda")[:, cols_dev].cpu().numpy()
     V = ctx.get_momentum(device="cuda")[:, cols_dev].cpu().numpy()
+    ctx.check_guards()
     ctx.close()
     torch.cuda.empty_cache()
     H.assert_close(X, orc.X, H.TOL_SAME_INPUT, name + " X")

@@ -50,11 +50,14 @@ def _run(B, w, steps, fused=True, norm="mean", order="mix_then_update", check_st
         else:
             g = H.to_device(payload)
             ld = {}
+        g_before = g.clone()
         if fused:
             ctx.step_fused(g, n, **ld)
         else:
             ctx.accumulate(g, n, **ld)
             ctx.step()
+        assert torch.equal(g.view(torch.int16) if g.dtype == torch.bfloat16 else g,
+                           g_before.view(torch.int16) if g.dtype == torch.bfloat16 else g_before)   # G is read-only
         orc.step(values, n.tolist())
         if orc_unr:
             orc_unr.step(unr, n.tolist())
@@ -74,6 +77,7 @@ def _run(B, w, steps, fused=True, norm="mean", order="mix_then_update", check_st
                 H.assert_close(X, orc_unr.X, H.TOL_BF16_ROUNDING, "%s step %d X vs un-rounded" % (w.name, t + 1))
             out[t + 1] = e
     assert ctx.get_step() == steps
+    ctx.check_guards()            # no kernel wrote outside X, V or the accumulator
     ctx.close()
     return out
 

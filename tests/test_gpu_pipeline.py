@@ -42,6 +42,7 @@ def _against_oracle(B, w, steps, counts=None, fused=True):
         orc.step(values, [int(v) for v in n])
     H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT, w.name)
     H.assert_close(ctx.get_momentum().numpy(), orc.V, H.TOL_SAME_INPUT, w.name)
+    ctx.check_guards()
     ctx.close()
     return launches
 
