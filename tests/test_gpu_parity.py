@@ -453,3 +453,30 @@ def test_matcha_with_optimised_per_matching_probabilities(B):
     assert len(seen) > 1
     H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
     ctx.close()
+
+
+def test_work_is_enqueued_on_the_callers_stream(B):
+    """Every entry point takes the stream to enqueue on: a run on a side stream (inputs produced on
+    that stream, no other synchronisation) equals the run on the default stream bit for bit."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg4_matcha_vgg16"], 6 * 512 + 8, steps=4)
+    x0 = torch.from_numpy(WL.init_params(w)).cuda()
+    ref = B.context_for(w)
+    ref.set_params(x0)
+    side = torch.cuda.Stream()
+    other = B.context_for(w)
+    payloads = [WL.gradients_np(w, t)[0] for t in range(w.steps)]
+    counts = [H.lib_counts(B, w, t) for t in range(w.steps)]
+    for t in range(w.steps):
+        ref.step_fused(H.to_device(payloads[t]), counts[t])
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        other.set_params(x0)
+        for t in range(w.steps):
+            g = H.to_device(payloads[t]) * 1.0            # produced on the side stream
+            other.step_fused(g, counts[t])
+        X = other.get_params(device="cuda")
+        V = other.get_momentum(device="cuda")
+    side.synchronize()
+    assert torch.equal(X, ref.get_params(device="cuda")) and torch.equal(V, ref.get_momentum(device="cuda"))
+    ref.close(); other.close()
