@@ -210,8 +210,10 @@ int nb_set_params(nb_ctx *c, const float *x0, int per_learner, void *stream);
 /* Masked accumulate (step 1): acc[i,p] = sum_{m < finished[i]} grads[i,m,p], fp32 accumulation in
  * ascending m; rows m >= finished[i] are never read.
  * grads: device, element (i,m,p) at grads[i*ld_k + m*ld_m + p], dtype NB_F32 or NB_BF16;
- * ld_m, ld_k in elements, 0 = dense (ld_m = P, ld_k = M*P).  The 128-bit path needs grads, ld_m
- * and ld_k aligned to 4 elements; anything else runs a scalar kernel on the GPU.
+ * ld_m, ld_k in elements, 0 = dense (ld_m = P, ld_k = M*P).  Alignment decides the kernel, never
+ * the result (all paths give identical bits): with grads 16-byte aligned and ld_m, ld_k multiples of
+ * 16 bytes the bulk-copy pipeline kernels cover all full 512-column tiles; with 4-element alignment
+ * the direct kernels use 128-bit / 64-bit loads; anything else runs scalar loads, still on the GPU.
  * finished: host [K], each in [0, M].  Errors: NB_ERR_ARG. */
 int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
                   const int32_t *finished, void *stream);
