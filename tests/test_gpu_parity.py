@@ -480,3 +480,14 @@ def test_work_is_enqueued_on_the_callers_stream(B):
     side.synchronize()
     assert torch.equal(X, ref.get_params(device="cuda")) and torch.equal(V, ref.get_momentum(device="cuda"))
     ref.close(); other.close()
+
+
+@pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16",
+                                  "cfg5_scale_ring"])
+def test_full_step_counts_of_the_configurations(B, name):
+    """The configurations' own step counts (50 / 50 / 20 / 20): tolerance checked at step 10 and at the last step."""
+    w = WL.WORKLOADS[name]
+    ws = WL.scaled(w, 2 * 512 + 72, steps=w.steps)
+    errs = _run(B, ws, ws.steps, fused=True, check_steps=(10, ws.steps), with_unrounded=(ws.grad_dtype == "bf16"))
+    assert set(errs) == {10, ws.steps}
+    assert all(e[0] < H.TOL_SAME_INPUT for e in errs.values())
