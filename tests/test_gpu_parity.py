@@ -491,3 +491,22 @@ def test_full_step_counts_of_the_configurations(B, name):
     errs = _run(B, ws, ws.steps, fused=True, check_steps=(10, ws.steps), with_unrounded=(ws.grad_dtype == "bf16"))
     assert set(errs) == {10, ws.steps}
     assert all(e[0] < H.TOL_SAME_INPUT for e in errs.values())
+
+
+def test_dense_mixing_matrix_at_the_table_limit(B):
+    """D-PSGD with the FULL topology and K = 32 fills the sparse table exactly (1024 non-zeros); it
+    must agree with the oracle's dense W (and, up to rounding order, with the all-reduce variant)."""
+    import torch
+    K, P, M = 32, 2 * 512 + 16, 2
+    rng = np.random.default_rng(32)
+    X0 = rng.standard_normal((K, P)).astype(np.float32)
+    ctx = B.NbContext(K, P, M, 0.1, 0.9, "dpsgd", B.make_topology("full"))
+    orc = O.Oracle(K, P, M, 0.1, 0.9, "dpsgd", W=O.full_W(K))
+    ctx.set_params(torch.from_numpy(X0).cuda(), per_learner=True); orc.set_params(X0)
+    for t in range(3):
+        G = rng.standard_normal((K, M, P)).astype(np.float32)
+        n = rng.integers(0, M + 1, K).tolist()
+        ctx.step_fused(torch.from_numpy(G).cuda(), n); orc.step(G, n)
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+    ctx.check_guards()
+    ctx.close()

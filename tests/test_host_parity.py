@@ -235,3 +235,19 @@ def test_per_matching_probabilities_drive_the_activation_words():
     bad, keep2 = B.make_topology("random_regular", degree=3, seed=1, alpha=0.1, act_probs=np.array([0.5, 1.5, 0.5, 0.5, 0.5]))
     Wbuf = np.zeros((K, K), dtype=np.float32)
     assert B.lib.nb_mixing_matrix(C.byref(bad), B.NB_MATCHA, K, 0, Wbuf.ctypes.data_as(C.POINTER(C.c_float)), None) == B.NB_ERR_ARG
+
+
+def test_table_limits_are_reported():
+    import ctypes as C
+    W = np.zeros((64, 64), dtype=np.float32)
+    Wp = W.ctypes.data_as(C.POINTER(C.c_float))
+    topo, _ = B.make_topology("full")
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_DPSGD, 32, 0, Wp, None) == B.NB_OK          # 1024 non-zeros: fits
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_DPSGD, 33, 0, Wp, None) == B.NB_ERR_UNSUPPORTED
+    assert B.lib.nb_mixing_matrix(None, B.NB_ALLREDUCE, 64, 0, Wp, None) == B.NB_OK               # the mean needs no table
+    assert B.lib.nb_mixing_matrix(None, B.NB_ALLREDUCE, 65, 0, Wp, None) == B.NB_ERR_UNSUPPORTED
+    # more matchings than activation bits
+    K = 4
+    partner = np.full((33, K), -1, dtype=np.int32)
+    topo, keep = B.make_topology("matchings", partner=partner, alpha=0.1, act_prob=0.5)
+    assert B.lib.nb_mixing_matrix(C.byref(topo), B.NB_MATCHA, K, 0, Wp, None) == B.NB_ERR_UNSUPPORTED
