@@ -51,6 +51,7 @@ def parse_args():
                     help="run the workload's sizes with another variant (dpsgd = ring)")
     ap.add_argument("--order", default="mix_then_update", choices=["mix_then_update", "update_then_mix"])
     ap.add_argument("--unfused", action="store_true", help="time nb_accumulate + nb_step instead of nb_step_fused")
+    ap.add_argument("--grad-pad", type=int, default=0, help="experiment: extra elements of row pitch in the gradient buffers")
     ap.add_argument("--cols", type=int, default=0, help="profiling aid: run the workload on this many columns instead of its P")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
@@ -218,6 +219,13 @@ def run_ours(args, w):
     free, _ = torch.cuda.mem_get_info()
     n_buf = 2 if free > 2 * g_bytes + 4 * w.K * w.P * 4 + (8 << 30) else 1
     bufs = [WL.gradients_torch(wr, b, dev) for b in range(n_buf)]
+    ld = {}
+    if args.grad_pad:
+        wide = [torch.empty((w.K, w.M, w.P + args.grad_pad), dtype=b.dtype, device=dev) for b in bufs]
+        for dst, src in zip(wide, bufs):
+            dst[:, :, :w.P].copy_(src)
+        bufs = [b[:, :, :w.P] for b in wide]
+        ld = dict(ld_m=w.P + args.grad_pad, ld_k=w.M * (w.P + args.grad_pad))
     gen = torch.Generator(device=dev)
     gen.manual_seed(wr.seed)
     x0 = torch.randn(w.P, generator=gen, device=dev, dtype=torch.float32) * w.init_sigma
@@ -228,10 +236,10 @@ def run_ours(args, w):
 
     def one_step(g, n):
         if args.unfused:
-            ctx.accumulate(g, n)
+            ctx.accumulate(g, n, **ld)
             ctx.step()
         else:
-            ctx.step_fused(g, n)
+            ctx.step_fused(g, n, **ld)
 
     def counts(t):
         return B.straggler_sample(w.straggler_model, w.seed, t, w.K, w.M, w.straggler_params)[0]

@@ -214,6 +214,7 @@ int nb_set_params(nb_ctx *c, const float *x0, int per_learner, void *stream);
  * the result (all paths give identical bits): with grads 16-byte aligned and ld_m, ld_k multiples of
  * 16 bytes the bulk-copy pipeline kernels cover all full 512-column tiles; with 4-element alignment
  * the direct kernels use 128-bit / 64-bit loads; anything else runs scalar loads, still on the GPU.
+ * (Rows whose pitch is a multiple of 2 KB stream 1-2 % faster than other 16-byte multiples.)
  * finished: host [K], each in [0, M].  Errors: NB_ERR_ARG. */
 int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
                   const int32_t *finished, void *stream);
