@@ -3,7 +3,6 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -267,7 +266,6 @@ int nb_create(nb_ctx **out, int K, int64_t P, int M, float lr, float mom, int va
   // Row pitch of X, V and acc: a multiple of the 512-column tile (2 KB), so that every row segment a
   // tile copies starts on a 2 KB boundary (measured: 2-3 % more bandwidth than 128-byte multiples).
   c->ldx = (P + 511) / 512 * 512;
-  if (const char *extra = std::getenv("NB_LDX_EXTRA")) c->ldx += 32 * (int64_t)std::atoi(extra);  // pitch experiments
   c->mx = mx;
 
   auto bail = [&](cudaError_t e, const char *what) {
