@@ -244,8 +244,10 @@ int nb_step_fused(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t
 /* As nb_step_fused with the gradient stream in HOST memory (pinned for speed): copies only the
  * finished mini-batch rows into a staging buffer the context allocates on first use ([K,M,P]
  * elements of the widest dtype seen), runs the fused step and, when mean_out is not NULL, writes
- * the mean model (Alg. 1 "Output") to host memory mean_out[P].  Waits for `stream` before it
- * returns. */
+ * the mean model (Alg. 1 "Output") to host memory mean_out[P].  The columns are processed in up to
+ * 8 chunks so that the host-to-device copies, the kernels and the device-to-host copy of the mean
+ * overlap (two internal streams and a few events are created on first use; the kernels run on
+ * `stream`).  Waits for all of it before it returns.  Same result as nb_step_fused, bit for bit. */
 int nb_step_fused_host(nb_ctx *c, const void *grads_host, int dtype, int64_t ld_m, int64_t ld_k,
                        const int32_t *finished, float *mean_out, void *stream);
 

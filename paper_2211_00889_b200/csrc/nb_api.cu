@@ -27,6 +27,10 @@ struct nb_ctx {
   int *d_err = nullptr;  // device word a kernel sets when one of its bounded waits runs out
   void *staging = nullptr;
   size_t staging_bytes = 0;
+  // nb_step_fused_host overlaps the copies of one column chunk with the kernels of the previous one
+  static constexpr int kHostChunks = 8;
+  cudaStream_t s_copy = nullptr, s_out = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_h2d[kHostChunks] = {nullptr}, ev_done[kHostChunks] = {nullptr};
   int64_t step = 0;
   bool acc_fresh = false, device_mix_valid = false;
   int32_t n_acc[NB_MAX_K] = {0};
@@ -189,21 +193,24 @@ int build_device_mixing(nb_ctx *c, cudaStream_t st) {
   return NB_OK;
 }
 
+// The step kernels on the columns `a` describes (all of them, or one chunk); the mixing matrix of
+// the current step must already be on the device.
+int launch_update(nb_ctx *c, const nb::StepArgs &a, int src, cudaStream_t st) {
+  int n_launched = 0;
+  cudaError_t e;
+  if (c->variant == NB_CENTRALIZED) e = nb::launch_centralized(a, src, c->d_err, &n_launched, st);
+  else e = nb::launch_step(a, src, c->d_err, &n_launched, &c->last_plan, st);
+  c->launches += n_launched;
+  if (e != cudaSuccess) return cuda_fail(c, e, "launch_step");
+  return NB_OK;
+}
+
 int run_update(nb_ctx *c, nb::StepArgs *a, int src, cudaStream_t st) {
   fill_update_args(c, a);
-  if (c->variant == NB_CENTRALIZED) {
-    int n_launched = 0;
-    cudaError_t e = nb::launch_centralized(*a, src, c->d_err, &n_launched, st);
-    c->launches += n_launched;
-    if (e != cudaSuccess) return cuda_fail(c, e, "launch_centralized");
-  } else {
-    int rc = build_device_mixing(c, st);
-    if (rc != NB_OK) return rc;
-    int n_launched = 0;
-    cudaError_t e = nb::launch_step(*a, src, c->d_err, &n_launched, &c->last_plan, st);
-    c->launches += n_launched;
-    if (e != cudaSuccess) return cuda_fail(c, e, "launch_step");
-  }
+  int rc = build_device_mixing(c, st);
+  if (rc != NB_OK) return rc;
+  rc = launch_update(c, *a, src, st);
+  if (rc != NB_OK) return rc;
   c->step++;
   c->acc_fresh = false;
   return NB_OK;
@@ -322,6 +329,13 @@ int nb_destroy(nb_ctx *c) {
   cudaFree(c->d_partner);
   cudaFree(c->d_err);
   cudaFree(c->staging);
+  if (c->s_copy) cudaStreamDestroy(c->s_copy);
+  if (c->s_out) cudaStreamDestroy(c->s_out);
+  if (c->ev_start) cudaEventDestroy(c->ev_start);
+  for (int q = 0; q < nb_ctx::kHostChunks; ++q) {
+    if (c->ev_h2d[q]) cudaEventDestroy(c->ev_h2d[q]);
+    if (c->ev_done[q]) cudaEventDestroy(c->ev_done[q]);
+  }
   cudaGetLastError();
   delete c;
   return NB_OK;
@@ -471,7 +485,7 @@ int nb_step_fused_host(nb_ctx *c, const void *grads_host, int dtype, int64_t ld_
   if (ld_m < c->P) return fail(c, NB_ERR_ARG, "ld_m is smaller than P");
   for (int i = 0; i < c->K; ++i)
     if (finished[i] < 0 || finished[i] > c->M) return fail(c, NB_ERR_ARG, "finished count outside [0, M]");
-  const int64_t ldg = (c->P + 31) / 32 * 32;  // staging pitch, elements
+  const int64_t ldg = (c->P + 511) / 512 * 512;  // staging pitch, elements: rows start on 2 KB boundaries
   const size_t need = (size_t)c->K * (size_t)c->M * (size_t)ldg * es;
   if (c->staging_bytes < need) {
     NB_CUDA(c, cudaStreamSynchronize(st));
@@ -481,19 +495,69 @@ int nb_step_fused_host(nb_ctx *c, const void *grads_host, int dtype, int64_t ld_
     NB_CUDA(c, cudaMalloc(&c->staging, need));
     c->staging_bytes = need;
   }
-  // only the finished mini-batches cross the bus: the abandoned ones are never needed
-  for (int i = 0; i < c->K; ++i)
-    for (int m = 0; m < finished[i]; ++m) {
-      const char *src = (const char *)grads_host + ((size_t)i * (size_t)ld_k + (size_t)m * (size_t)ld_m) * es;
-      char *dst = (char *)c->staging + ((size_t)i * (size_t)c->M + (size_t)m) * (size_t)ldg * es;
-      NB_CUDA(c, cudaMemcpyAsync(dst, src, (size_t)c->P * es, cudaMemcpyHostToDevice, st));
+  if (mean_out && !c->d_mean) NB_CUDA(c, cudaMalloc(&c->d_mean, sizeof(float) * (size_t)c->P));
+  if (!c->s_copy) {
+    NB_CUDA(c, cudaStreamCreateWithFlags(&c->s_copy, cudaStreamNonBlocking));
+    NB_CUDA(c, cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking));
+    NB_CUDA(c, cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming));
+    for (int q = 0; q < nb_ctx::kHostChunks; ++q) {
+      NB_CUDA(c, cudaEventCreateWithFlags(&c->ev_h2d[q], cudaEventDisableTiming));
+      NB_CUDA(c, cudaEventCreateWithFlags(&c->ev_done[q], cudaEventDisableTiming));
     }
-  int rc = nb_step_fused(c, c->staging, dtype, ldg, (int64_t)c->M * ldg, finished, stream);
-  if (rc != NB_OK) return rc;
-  if (mean_out) {
-    rc = nb_get_mean_params(c, mean_out, stream);
-    if (rc != NB_OK) return rc;
   }
+  nb::StepArgs a;
+  int esz = 4;
+  int rc = fill_step_args(c, c->staging, dtype, ldg, (int64_t)c->M * ldg, finished, &a, &esz);
+  if (rc != NB_OK) return rc;
+  record_stats(c, a, esz);
+  fill_update_args(c, &a);
+  rc = build_device_mixing(c, st);
+  if (rc != NB_OK) return rc;
+  const int src_kind = dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16;
+  // Column chunks (multiples of the 512-column tile, at least 64K columns each): the copy stream
+  // brings chunk q+1 over the bus while `stream` runs the kernels of chunk q and the output stream
+  // returns chunk q-1's mean model; the three directions overlap because columns are independent.
+  int n_chunks = (int)(c->P / 65536);
+  if (n_chunks > nb_ctx::kHostChunks) n_chunks = nb_ctx::kHostChunks;
+  if (n_chunks < 1) n_chunks = 1;
+  const int64_t per_chunk = ((c->P / n_chunks) + 511) / 512 * 512;
+  NB_CUDA(c, cudaEventRecord(c->ev_start, st));
+  NB_CUDA(c, cudaStreamWaitEvent(c->s_copy, c->ev_start, 0));  // the staging buffer is free once `stream` got here
+  for (int q = 0; q < n_chunks; ++q) {
+    const int64_t c0 = (int64_t)q * per_chunk;
+    const int64_t cols = (q == n_chunks - 1) ? c->P - c0 : per_chunk;
+    if (cols <= 0) break;
+    // only the finished mini-batches cross the bus: the abandoned ones are never needed.  One
+    // pitched copy per learner moves its n_i row segments (row by row when the pitch is too large).
+    for (int i = 0; i < c->K; ++i) {
+      if (finished[i] == 0) continue;
+      const char *src = (const char *)grads_host + ((size_t)i * (size_t)ld_k + (size_t)c0) * es;
+      char *dst = (char *)c->staging + ((size_t)i * (size_t)c->M * (size_t)ldg + (size_t)c0) * es;
+      const size_t spitch = (size_t)ld_m * es, dpitch = (size_t)ldg * es;
+      if (spitch < (size_t)2147483647 && dpitch < (size_t)2147483647) {
+        NB_CUDA(c, cudaMemcpy2DAsync(dst, dpitch, src, spitch, (size_t)cols * es, (size_t)finished[i],
+                                     cudaMemcpyHostToDevice, c->s_copy));
+      } else {
+        for (int m = 0; m < finished[i]; ++m)
+          NB_CUDA(c, cudaMemcpyAsync(dst + (size_t)m * dpitch, src + (size_t)m * spitch, (size_t)cols * es,
+                                     cudaMemcpyHostToDevice, c->s_copy));
+      }
+    }
+    NB_CUDA(c, cudaEventRecord(c->ev_h2d[q], c->s_copy));
+    NB_CUDA(c, cudaStreamWaitEvent(st, c->ev_h2d[q], 0));
+    rc = launch_update(c, nb::column_range(a, c0, cols, esz), src_kind, st);
+    if (rc != NB_OK) return rc;
+    if (mean_out) {
+      NB_CUDA(c, nb::launch_mean(c->X + c0, c->ldx, c->rows, cols, c->d_mean + c0, st));
+      c->launches++;
+      NB_CUDA(c, cudaEventRecord(c->ev_done[q], st));
+      NB_CUDA(c, cudaStreamWaitEvent(c->s_out, c->ev_done[q], 0));
+      NB_CUDA(c, cudaMemcpyAsync(mean_out + c0, c->d_mean + c0, sizeof(float) * (size_t)cols, cudaMemcpyDeviceToHost, c->s_out));
+    }
+  }
+  c->step++;
+  c->acc_fresh = false;
+  NB_CUDA(c, cudaStreamSynchronize(c->s_out));
   return check_device_error(c, st);
 }
 

@@ -268,15 +268,7 @@ cudaError_t configure_kernels() {
 namespace {
 // Column range [done, P) of the same problem: what the direct-load kernels take over after a
 // pipeline kernel has covered the full tiles.
-StepArgs tail_of(const StepArgs &a, int64_t done, int es) {
-  StepArgs r = a;
-  r.X += done;
-  r.V += done;
-  r.acc += done;
-  r.G = reinterpret_cast<const unsigned char *>(a.G) + done * es;
-  r.P = a.P - done;
-  return r;
-}
+StepArgs tail_of(const StepArgs &a, int64_t done, int es) { return column_range(a, done, a.P - done, es); }
 // The accumulator presented as a one-row fp32 gradient stream (0 + acc == acc bit for bit: acc is never -0).
 StepArgs acc_as_stream(const StepArgs &a) {
   StepArgs p = a;
@@ -288,6 +280,16 @@ StepArgs acc_as_stream(const StepArgs &a) {
   return p;
 }
 }  // namespace
+
+StepArgs column_range(const StepArgs &a, int64_t c0, int64_t cols, int es) {
+  StepArgs r = a;
+  r.X += c0;
+  r.V += c0;
+  r.acc += c0;
+  if (a.G) r.G = reinterpret_cast<const unsigned char *>(a.G) + c0 * es;
+  r.P = cols;
+  return r;
+}
 
 cudaError_t launch_accumulate(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st) {
   *launches = 0;

@@ -61,6 +61,10 @@ cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, 
 cudaError_t configure_pipeline();
 cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan, int *err_flag, cudaStream_t st);
 
+// The same problem restricted to columns [c0, c0 + cols): every step of the path is independent per
+// column, so a column range is a complete problem of its own (es = bytes per gradient element).
+StepArgs column_range(const StepArgs &a, int64_t c0, int64_t cols, int es);
+
 int step_threads_per_block(const StepArgs &a);
 // Masked accumulate on all P columns (pipeline kernel on the full tiles when it applies).
 cudaError_t launch_accumulate(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st);

@@ -510,3 +510,30 @@ def test_dense_mixing_matrix_at_the_table_limit(B):
     H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
     ctx.check_guards()
     ctx.close()
+
+
+@pytest.mark.parametrize("name", ["cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16", "cfg2_allreduce_resnet18"])
+def test_host_buffer_entry_point_in_several_chunks(B, name):
+    """Enough columns for nb_step_fused_host to split the work into overlapped column chunks: the
+    result must equal nb_step_fused on the same values, bit for bit, mean model included."""
+    import torch
+    w = replace(WL.scaled(WL.WORKLOADS[name], 3 * 65536 + 520, steps=2), K=4, M=3)
+    if w.variant == "matcha":
+        w = replace(w, degree=3)
+    a, b = B.context_for(w), B.context_for(w)
+    gen = torch.Generator(device="cuda"); gen.manual_seed(5)
+    x0 = torch.randn(w.P, generator=gen, device="cuda") * 0.01
+    a.set_params(x0); b.set_params(x0)
+    mean = torch.empty(w.P, dtype=torch.float32).pin_memory()
+    for t in range(w.steps):
+        g = WL.gradients_torch(w, t, "cuda")
+        host = torch.empty(g.shape, dtype=g.dtype).pin_memory()
+        host.copy_(g)
+        n = np.array([3, 1, 0, 2]) if t == 0 else np.array([2, 3, 3, 1])
+        a.step_fused_host(host, n, mean_out=mean)
+        b.step_fused(g, n)
+        assert torch.equal(mean, b.get_mean_params())
+    assert a.get_step() == b.get_step() == w.steps
+    assert torch.equal(a.get_params(), b.get_params()) and torch.equal(a.get_momentum(), b.get_momentum())
+    a.check_guards()
+    a.close(); b.close()
