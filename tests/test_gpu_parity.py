@@ -537,3 +537,33 @@ def test_host_buffer_entry_point_in_several_chunks(B, name):
     assert torch.equal(a.get_params(), b.get_params()) and torch.equal(a.get_momentum(), b.get_momentum())
     a.check_guards()
     a.close(); b.close()
+
+
+def test_learning_rate_can_change_between_steps(B):
+    """nb_set_lr (e.g. a decay schedule as in Sec. 6.1): each step uses the rate set before it."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 2 * 512 + 8, steps=4)
+    ctx = B.context_for(w)
+    orc = H.oracle_for(w, w.P)
+    x0 = WL.init_params(w)
+    ctx.set_params(torch.from_numpy(x0).cuda()); orc.set_params(x0)
+    for t, lr in enumerate([0.8, 0.8, 0.08, 0.008]):
+        ctx.set_lr(lr)
+        orc.lr = lr
+        n = H.lib_counts(B, w, t)
+        payload, values = WL.gradients_np(w, t)
+        ctx.step_fused(H.to_device(payload), n)
+        orc.step(values, n.tolist())
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+    ctx.close()
+
+
+def test_reported_mixing_matrices(B):
+    for name in ("cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50"):
+        w = WL.scaled(WL.WORKLOADS[name], 64, steps=1)
+        ctx = B.context_for(w)
+        want = O.full_W(w.K) if w.variant == "allreduce" else O.ring_W(w.K)
+        assert np.abs(ctx.get_W(0).astype(np.float64) - want).max() < 1e-7
+        with pytest.raises(B.NbError):
+            ctx.get_matcha_activation(0)           # not a MATCHA context
+        ctx.close()
