@@ -131,6 +131,35 @@ struct PipeArgs {
   alignas(64) CUtensorMap gmap[kMaxRowsPerItem];  // G as [K, M, units]: box = (256, r, 1), r = 1..R
 };
 
+// acc += row_0 + row_1 + ... (ascending, one add at a time) over N rows `stride` bytes apart; all
+// loads are issued before the first add.  Same sequence of fp32 additions as a plain loop.
+template <int SRC, int N>
+__device__ __forceinline__ float4 sum_rows_n(float4 acc, const unsigned char *rowp, int stride) {
+  Raw<SRC> raw[N];
+#pragma unroll
+  for (int r = 0; r < N; ++r) {
+    if constexpr (SRC == kSrcBF16) raw[r].r = *reinterpret_cast<const uint2 *>(rowp + r * stride);
+    else raw[r].r = *reinterpret_cast<const float4 *>(rowp + r * stride);
+  }
+#pragma unroll
+  for (int r = 0; r < N; ++r) acc = add4(acc, widen(raw[r]));
+  return acc;
+}
+template <int SRC>
+__device__ __forceinline__ float4 sum_rows(float4 acc, const unsigned char *rowp, int stride, int rows) {
+  switch (rows) {
+    case 0: return acc;
+    case 1: return sum_rows_n<SRC, 1>(acc, rowp, stride);
+    case 2: return sum_rows_n<SRC, 2>(acc, rowp, stride);
+    case 3: return sum_rows_n<SRC, 3>(acc, rowp, stride);
+    case 4: return sum_rows_n<SRC, 4>(acc, rowp, stride);
+    case 5: return sum_rows_n<SRC, 5>(acc, rowp, stride);
+    case 6: return sum_rows_n<SRC, 6>(acc, rowp, stride);
+    case 7: return sum_rows_n<SRC, 7>(acc, rowp, stride);
+    default: return sum_rows_n<SRC, 8>(acc, rowp, stride);
+  }
+}
+
 struct PipeLayout {
   int32_t off_tab, off_xs, off_slots, slot_bytes, total;
 };
@@ -151,12 +180,13 @@ __host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, i
 }
 
 // ES = bytes per gradient element (2: bf16, 4: fp32).
-template <int ES, bool MEAN>
+// TT = tile width known at compile time (512, the usual shape: strides become immediates) or 0 (a.T).
+template <int ES, bool MEAN, int TT>
 __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeline_kernel(const __grid_constant__ PipeArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
   const StepArgs &s = a.s;
-  const int K = s.K, T = a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
+  const int K = s.K, T = TT ? TT : a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
   const int NSG = NS / NG;  // slots in each group's ring
   const PipeLayout L = pipe_layout(K, T, ES, R, NS, s.mix_slots);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);
@@ -281,13 +311,7 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
             if (!ok) break;
             const unsigned char *src = slots + (size_t)sl * L.slot_bytes;
             if (m0 == 0) v = reinterpret_cast<const float4 *>(src)[cq];
-            const unsigned char *rowp = src + T * 4 + (size_t)cq * 4 * ES;
-            for (int r = 0; r < rows; ++r) {
-              Raw<SRC> raw;
-              if constexpr (ES == 2) raw.r = *reinterpret_cast<const uint2 *>(rowp + (size_t)r * T * ES);
-              else raw.r = *reinterpret_cast<const float4 *>(rowp + (size_t)r * T * ES);
-              acc = add4(acc, widen(raw));
-            }
+            acc = sum_rows<SRC>(acc, src + T * 4 + cq * 4 * ES, T * ES, rows);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[sl]);
             if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
@@ -655,7 +679,10 @@ cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, 
 cudaError_t configure_pipeline() {
   cudaError_t e;
 #define NB_CFG(ES, MEAN)                                                                              \
-  if ((e = cudaFuncSetAttribute(nb_step_pipeline_kernel<ES, MEAN>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+  if ((e = cudaFuncSetAttribute(nb_step_pipeline_kernel<ES, MEAN, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                kSmemBudget)) != cudaSuccess)                                         \
+    return e;                                                                                         \
+  if ((e = cudaFuncSetAttribute(nb_step_pipeline_kernel<ES, MEAN, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                 kSmemBudget)) != cudaSuccess)                                         \
     return e;
   NB_CFG(2, true) NB_CFG(2, false) NB_CFG(4, true) NB_CFG(4, false)
@@ -691,13 +718,19 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
   }
   if (!encode_gmaps(&p, a, es, plan)) return cudaErrorInvalidValue;  // G: [K, M, units]; one map per box height
   const int threads = 32 + plan.n_groups * (32 + plan.T / 4);  // X producer + per group: producer warp + consumers
+#define NB_LAUNCH(ES, MEAN)                                                                                   \
+  do {                                                                                                        \
+    if (plan.T == 512) nb_step_pipeline_kernel<ES, MEAN, 512><<<plan.grid, threads, plan.smem_bytes, st>>>(p); \
+    else nb_step_pipeline_kernel<ES, MEAN, 0><<<plan.grid, threads, plan.smem_bytes, st>>>(p);                 \
+  } while (0)
   if (es == 2) {
-    if (a.mean_mode) nb_step_pipeline_kernel<2, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
-    else nb_step_pipeline_kernel<2, false><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
+    if (a.mean_mode) NB_LAUNCH(2, true);
+    else NB_LAUNCH(2, false);
   } else {
-    if (a.mean_mode) nb_step_pipeline_kernel<4, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
-    else nb_step_pipeline_kernel<4, false><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
+    if (a.mean_mode) NB_LAUNCH(4, true);
+    else NB_LAUNCH(4, false);
   }
+#undef NB_LAUNCH
   return cudaGetLastError();
 }
 
