@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <utility>
 #include <string>
 
 #include "nb_internal.h"
@@ -21,6 +22,10 @@ struct nb_ctx {
   // X, V and acc sit between guard bands (kGuardBytes of a fixed byte pattern before and after);
   // nb_check_guards verifies that no kernel wrote outside its arrays.
   unsigned char *X_base = nullptr, *V_base = nullptr, *acc_base = nullptr;
+  // second model array for the out-of-place step (allocated the first time that kernel is needed);
+  // after such a step X and X2 trade places
+  float *X2 = nullptr;
+  unsigned char *X2_base = nullptr;
   size_t model_bytes = 0, acc_bytes = 0;
   nb::MixTable *d_mix = nullptr;
   int32_t *d_partner = nullptr;
@@ -195,11 +200,29 @@ int build_device_mixing(nb_ctx *c, cudaStream_t st) {
 
 // The step kernels on the columns `a` describes (all of them, or one chunk); the mixing matrix of
 // the current step must already be on the device.
-int launch_update(nb_ctx *c, const nb::StepArgs &a, int src, cudaStream_t st) {
+int launch_update(nb_ctx *c, const nb::StepArgs &a, int src, cudaStream_t st, bool whole_range = false) {
   int n_launched = 0;
   cudaError_t e;
-  if (c->variant == NB_CENTRALIZED) e = nb::launch_centralized(a, src, c->d_err, &n_launched, st);
-  else e = nb::launch_step(a, src, c->d_err, &n_launched, &c->last_plan, st);
+  if (c->variant == NB_CENTRALIZED) {
+    e = nb::launch_centralized(a, src, c->d_err, &n_launched, st);
+  } else if (whole_range && nb::prefers_out_of_place(a, src)) {
+    // rows the bulk-copy kernel cannot take: read the old models from X, write the new ones to X2, swap
+    if (!c->X2) {
+      cudaError_t ea = alloc_guarded(&c->X2_base, &c->X2, c->model_bytes);
+      if (ea != cudaSuccess) return cuda_fail(c, ea, "cudaMalloc(X2)");
+    }
+    nb::StepArgs b = a;
+    b.X_out = c->X2;
+    e = nb::launch_step_out_of_place(b, src, st);
+    n_launched = 1;
+    c->last_plan = nb::PipePlan{};
+    if (e == cudaSuccess) {
+      std::swap(c->X, c->X2);
+      std::swap(c->X_base, c->X2_base);
+    }
+  } else {
+    e = nb::launch_step(a, src, c->d_err, &n_launched, &c->last_plan, st);
+  }
   c->launches += n_launched;
   if (e != cudaSuccess) return cuda_fail(c, e, "launch_step");
   return NB_OK;
@@ -209,7 +232,7 @@ int run_update(nb_ctx *c, nb::StepArgs *a, int src, cudaStream_t st) {
   fill_update_args(c, a);
   int rc = build_device_mixing(c, st);
   if (rc != NB_OK) return rc;
-  rc = launch_update(c, *a, src, st);
+  rc = launch_update(c, *a, src, st, true);
   if (rc != NB_OK) return rc;
   c->step++;
   c->acc_fresh = false;
@@ -322,6 +345,7 @@ int nb_destroy(nb_ctx *c) {
   DeviceGuard guard(c->device);
   cudaDeviceSynchronize();
   cudaFree(c->X_base);
+  cudaFree(c->X2_base);
   cudaFree(c->V_base);
   cudaFree(c->acc_base);
   cudaFree(c->d_mean);
@@ -657,8 +681,10 @@ int nb_check_guards(nb_ctx *c, void *stream) {
   cudaStream_t st = (cudaStream_t)stream;
   unsigned char h[2 * kGuardBytes];
   struct Arr { const char *name; unsigned char *base; size_t bytes; };
-  const Arr arrs[3] = {{"X", c->X_base, c->model_bytes}, {"V", c->V_base, c->model_bytes}, {"acc", c->acc_base, c->acc_bytes}};
+  const Arr arrs[4] = {{"X", c->X_base, c->model_bytes}, {"V", c->V_base, c->model_bytes}, {"acc", c->acc_base, c->acc_bytes},
+                       {"X (second array)", c->X2_base, c->model_bytes}};
   for (const Arr &a : arrs) {
+    if (!a.base) continue;
     NB_CUDA(c, cudaMemcpyAsync(h, a.base, kGuardBytes, cudaMemcpyDeviceToHost, st));
     NB_CUDA(c, cudaMemcpyAsync(h + kGuardBytes, a.base + kGuardBytes + a.bytes, kGuardBytes, cudaMemcpyDeviceToHost, st));
     NB_CUDA(c, cudaStreamSynchronize(st));

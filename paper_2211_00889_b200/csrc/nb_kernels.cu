@@ -161,6 +161,55 @@ __global__ void __launch_bounds__(256) nb_step_kernel(const __grid_constant__ St
 }
 
 // -------------------------------------------------------------------------------------------------
+// Out-of-place form of the sparse-W step in the Alg. 2 order: x_i(new) = sum_j W_ij x_j(old) - lr v_i
+// with the old models read straight from X (the neighbours' tiles hit in L1/L2: the same CTA touches
+// them within a few microseconds) and the new ones written to X_out.  No staging, hence no shared
+// memory beyond the W table and full occupancy.  Used when the bulk-copy kernel cannot take the
+// stream (rows that are not 16-byte aligned).  Same operation sequence as nb_step_kernel.
+// -------------------------------------------------------------------------------------------------
+template <int SRC, bool ALIGNED>
+__global__ void __launch_bounds__(256) nb_step_out_of_place_kernel(const __grid_constant__ StepArgs a) {
+  extern __shared__ float4 smem[];
+  const int tid = threadIdx.x, tpb = blockDim.x, K = a.K;
+  int32_t *s_col = reinterpret_cast<int32_t *>(smem);
+  float *s_val = reinterpret_cast<float *>(s_col + a.mix_slots);
+  int32_t *s_beg = reinterpret_cast<int32_t *>(s_val + a.mix_slots);
+  int32_t *s_end = s_beg + K;
+  for (int e = tid; e < a.mix_slots; e += tpb) {
+    s_col[e] = a.mix->col[e];
+    s_val[e] = a.mix->val[e];
+  }
+  for (int e = tid; e < K; e += tpb) {
+    s_beg[e] = a.mix->row_beg[e];
+    s_end[e] = a.mix->row_end[e];
+  }
+  __syncthreads();
+  const int64_t col0 = ((int64_t)blockIdx.x * tpb + tid) * kColsPerThread;
+  if (col0 >= a.P) return;
+  const int nvalid = (a.P - col0 < 4) ? (int)(a.P - col0) : 4;
+  const float *Xin = a.X + col0;
+  float *Xout = a.X_out + col0;
+  float *Vc = a.V + col0;
+  const int64_t ldx = a.ldx;
+  for (int i = 0; i < K; ++i) {
+    const float4 v = ld4(Vc + (int64_t)i * ldx);
+    const float4 g = gather<SRC, ALIGNED>(a, i, col0, nvalid);
+    const float4 vn = momentum(a.mom, v, a.s[i], g);
+    float4 xh = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int e = s_beg[i]; e < s_end[i]; ++e) {
+      const float w = s_val[e];
+      const float4 x = __ldg(reinterpret_cast<const float4 *>(Xin + (int64_t)s_col[e] * ldx));
+      xh.x = __fmaf_rn(w, x.x, xh.x);
+      xh.y = __fmaf_rn(w, x.y, xh.y);
+      xh.z = __fmaf_rn(w, x.z, xh.z);
+      xh.w = __fmaf_rn(w, x.w, xh.w);
+    }
+    st4(Vc + (int64_t)i * ldx, vn);
+    st4(Xout + (int64_t)i * ldx, descend(xh, a.lr, vn));
+  }
+}
+
+// -------------------------------------------------------------------------------------------------
 // Non-blocking synchronous centralized step (Alg. 3): one shared model.
 //   g = (1/K) sum_i s_i acc_i ; v <- mom v + g ; x <- x - lr v
 // -------------------------------------------------------------------------------------------------
@@ -324,6 +373,9 @@ cudaError_t launch_accumulate_direct_only(const StepArgs &a, int src, cudaStream
   return cudaGetLastError();
 }
 
+namespace {
+StepArgs acc_as_stream(const StepArgs &a);
+}
 static cudaError_t launch_step_direct(const StepArgs &a, int src, cudaStream_t st) {
   if (src == kSrcAcc) return launch_step_t<kSrcAcc, true>(a, st);
   if (src == kSrcF32) return a.g_aligned ? launch_step_t<kSrcF32, true>(a, st) : launch_step_t<kSrcF32, false>(a, st);
@@ -331,6 +383,27 @@ static cudaError_t launch_step_direct(const StepArgs &a, int src, cudaStream_t s
 }
 
 cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st) { return launch_step_direct(a, src, st); }
+
+bool prefers_out_of_place(const StepArgs &a, int src) {
+  if (a.mean_mode || a.order != NB_ORDER_MIX_THEN_UPDATE) return false;
+  const int es = src == kSrcBF16 ? 2 : 4;
+  const StepArgs p = src == kSrcAcc ? acc_as_stream(a) : a;
+  PipePlan plan;
+  return !plan_pipeline(p, es, &plan);
+}
+
+cudaError_t launch_step_out_of_place(const StepArgs &a, int src, cudaStream_t st) {
+  const int tpb = 256;
+  const int64_t per_block = (int64_t)tpb * kColsPerThread;
+  const unsigned grid = (unsigned)((a.P + per_block - 1) / per_block);
+  const size_t smem = (size_t)a.mix_slots * 8 + (size_t)a.K * 8;
+#define NB_OOP(SRC, AL) nb_step_out_of_place_kernel<SRC, AL><<<grid, tpb, smem, st>>>(a)
+  if (src == kSrcAcc) NB_OOP(kSrcAcc, true);
+  else if (src == kSrcF32) { if (a.g_aligned) NB_OOP(kSrcF32, true); else NB_OOP(kSrcF32, false); }
+  else { if (a.g_aligned) NB_OOP(kSrcBF16, true); else NB_OOP(kSrcBF16, false); }
+#undef NB_OOP
+  return cudaGetLastError();
+}
 
 cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, PipePlan *used, cudaStream_t st) {
   *launches = 0;
