@@ -202,3 +202,35 @@ def test_accumulate_on_pipeline_sizes(B, dtype, M):
     H.assert_close(acc.numpy(), O.accumulate(G.float().cpu().numpy(), n.tolist()), 2e-6)
     assert float(acc[0].abs().max()) == 0.0
     a.close(); b.close()
+
+
+def test_in_place_and_out_of_place_steps_interleave(B):
+    """A context may see aligned streams (in-place pipeline kernel) and unaligned ones (out-of-place
+    kernel, after which the two model arrays trade places) in any order; state and results must be
+    those of a context that only ever saw aligned streams."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg5_scale_ring"], 4 * 512 + 40, steps=6)
+    ref, mix = B.context_for(w), B.context_for(w)
+    x0 = torch.from_numpy(WL.init_params(w)).cuda()
+    ref.set_params(x0); mix.set_params(x0)
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        g = H.to_device(WL.gradients_np(w, t)[0])
+        ref.step_fused(g, n)
+        if t in (1, 2, 4):                                   # unaligned view of the same values
+            flat = torch.empty(g.numel() + 1, dtype=g.dtype, device="cuda")
+            shifted = flat[1:].view_as(g)
+            shifted.copy_(g)
+            mix.step_fused(shifted, n)
+            assert mix.get_kernel_plan()["pipeline"] == 0
+        else:
+            mix.step_fused(g, n)
+            assert mix.get_kernel_plan()["pipeline"] == 1
+        if t == 2:                                           # checkpoint right after a swap
+            X, V, step = mix.get_params(), mix.get_momentum(), mix.get_step()
+            mix.set_state(step, X, V)
+        assert torch.equal(ref.get_params(), mix.get_params())
+    assert torch.equal(ref.get_momentum(), mix.get_momentum())
+    assert torch.equal(ref.get_mean_params(), mix.get_mean_params())
+    mix.check_guards()
+    ref.close(); mix.close()
