@@ -215,6 +215,9 @@ int nb_set_params(nb_ctx *c, const float *x0, int per_learner, void *stream);
  * 16 bytes the bulk-copy pipeline kernels cover all full 512-column tiles; with 4-element alignment
  * the direct kernels use 128-bit / 64-bit loads; anything else runs scalar loads, still on the GPU.
  * (Rows whose pitch is a multiple of 2 KB stream 1-2 % faster than other 16-byte multiples.)
+ * With a sparse W, rows that are not 16-byte aligned are handled out of place: the first such
+ * step allocates a second [K,P] model array (NB_ERR_NOMEM if that fails) and the two arrays trade
+ * places after every such step; nothing changes for the caller.
  * finished: host [K], each in [0, M].  Errors: NB_ERR_ARG. */
 int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
                   const int32_t *finished, void *stream);
