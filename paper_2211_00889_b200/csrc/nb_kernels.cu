@@ -346,10 +346,15 @@ cudaError_t launch_accumulate(const StepArgs &a, int src, int *err_flag, int *la
   PipePlan plan;
   int64_t done = 0;
   if (plan_stream(a, es, false, &plan)) {
+    // cudaErrorNotSupported: the driver refused a tensor map for this memory (nothing was launched);
+    // the direct-load kernel then takes the whole range
     cudaError_t e = launch_stream_pipeline(a, es, false, plan, err_flag, st);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-    done = (int64_t)plan.n_tiles * plan.T;
+    if (e == cudaSuccess) {
+      ++*launches;
+      done = (int64_t)plan.n_tiles * plan.T;
+    } else if (e != cudaErrorNotSupported) {
+      return e;
+    }
   }
   if (done < a.P) {
     cudaError_t e = launch_accumulate_direct_only(tail_of(a, done, es), src, st);
@@ -415,10 +420,13 @@ cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches
   int64_t done = 0;
   if (plan_pipeline(p, es, &plan)) {
     cudaError_t e = launch_step_pipeline(p, es, plan, err_flag, st);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-    *used = plan;
-    done = (int64_t)plan.n_tiles * plan.T;
+    if (e == cudaSuccess) {
+      ++*launches;
+      *used = plan;
+      done = (int64_t)plan.n_tiles * plan.T;
+    } else if (e != cudaErrorNotSupported) {  // NotSupported: no tensor map for this memory, nothing launched
+      return e;
+    }
   }
   if (done < a.P) {  // ragged tail (or everything, when the pipeline does not apply)
     cudaError_t e = launch_step_direct(tail_of(a, done, es), src, st);
@@ -451,9 +459,12 @@ cudaError_t launch_centralized(const StepArgs &a, int src, int *err_flag, int *l
   int64_t done = 0;
   if (plan_stream(p, es, true, &plan)) {
     cudaError_t e = launch_stream_pipeline(p, es, true, plan, err_flag, st);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-    done = (int64_t)plan.n_tiles * plan.T;
+    if (e == cudaSuccess) {
+      ++*launches;
+      done = (int64_t)plan.n_tiles * plan.T;
+    } else if (e != cudaErrorNotSupported) {
+      return e;
+    }
   }
   if (done < a.P) {
     cudaError_t e = launch_centralized_direct(tail_of(a, done, es), src, st);

@@ -668,7 +668,7 @@ cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, 
   p.n_tiles = plan.n_tiles;
   p.n_groups = plan.n_groups;
   p.err = err_flag;
-  if (!encode_gmaps(&p, a, es, plan)) return cudaErrorInvalidValue;
+  if (!encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;  // nothing launched: caller falls back
   const int threads = plan.n_groups * (32 + plan.T / 4);
   if (es == 2) {
     if (centralized) nb_stream_pipeline_kernel<2, kModeCentralized><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
@@ -718,9 +718,9 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
     const cuuint32_t xbox[2] = {kBoxInner, (cuuint32_t)a.K};
     const cuuint32_t vbox[2] = {kBoxInner, 1};
     if (!encode_map(&p.xmap, a.X, ub, 2, dims, strides, xbox) || !encode_map(&p.vmap, a.V, ub, 2, dims, strides, vbox))
-      return cudaErrorInvalidValue;
+      return cudaErrorNotSupported;  // nothing launched: caller falls back to the direct-load kernel
   }
-  if (!encode_gmaps(&p, a, es, plan)) return cudaErrorInvalidValue;  // G: [K, M, units]; one map per box height
+  if (!encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;  // G: [K, M, units]; one map per box height
   const int threads = 32 + plan.n_groups * (32 + plan.T / 4);  // X producer + per group: producer warp + consumers
 #define NB_LAUNCH(ES, MEAN)                                                                                   \
   do {                                                                                                        \
