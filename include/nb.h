@@ -287,6 +287,14 @@ int nb_get_stats(const nb_ctx *c, int64_t *sum_finished, double *algorithmic_byt
  * that ran out, NB_OK otherwise. */
 int nb_check_guards(nb_ctx *c, void *stream);
 
+/* Self-test of the kernels' bounded waits: runs one warp that waits, with a limit of about a
+ * millisecond, on a barrier nothing will complete, and checks that every lane gave up, that the
+ * device error word carried the wait's code and that the kernel returned normally.  The error word
+ * is cleared again: the context stays usable.  Waits for `stream`.  NB_OK if all of that held,
+ * NB_ERR_STATE otherwise.  (The waits of the production kernels use the same code with a limit of
+ * about a second; when one runs out the context reports a sticky NB_ERR_CUDA.) */
+int nb_selftest_wait_timeout(nb_ctx *c, void *stream);
+
 /* Which kernel shape ran the most recent step (for reports and tests), host out plan[8]:
  * [0] 1 if the bulk-copy pipeline kernel covered the full tiles, 0 if the direct-load kernel did
  * everything; [1] tile width in columns; [2] consumer groups per CTA; [3] ring slots per CTA;

@@ -90,6 +90,7 @@ def _load():
         "nb_runtime_report_compute": [P(nb_straggler), i32, i32, i64, i64, P(nb_runtime_report)],
         "nb_get_kernel_plan": [vp, P(C.c_int32)],
         "nb_check_guards": [vp, vp],
+        "nb_selftest_wait_timeout": [vp, vp],
         "nb_step_static": [i32, i64, i32, f32, f32, vp, vp, i64, vp, i32, i64, i64, P(C.c_int32), vp],
     }
     for name, args in sig.items():
@@ -106,7 +107,7 @@ EXPORTED = ["nb_straggler_sample", "nb_topology_matchings", "nb_mixing_matrix", 
             "nb_last_error", "nb_set_option", "nb_set_lr", "nb_set_params", "nb_accumulate", "nb_step",
             "nb_step_fused", "nb_step_fused_host", "nb_get_params", "nb_get_momentum", "nb_get_accumulator",
             "nb_get_mean_params", "nb_set_state", "nb_get_step", "nb_get_W", "nb_get_matcha_activation",
-            "nb_get_device_mixing", "nb_get_stats", "nb_step_static", "nb_get_kernel_plan", "nb_check_guards",
+            "nb_get_device_mixing", "nb_get_stats", "nb_step_static", "nb_get_kernel_plan", "nb_check_guards", "nb_selftest_wait_timeout",
             "nb_matcha_optimize", "nb_begin_iteration", "nb_accumulate_minibatch", "nb_get_finished", "nb_runtime_report_compute"]
 
 
@@ -359,6 +360,9 @@ class NbContext:
         b = C.c_uint32(0)
         self._ck(lib.nb_get_device_mixing(self._h, C.byref(b), W.ctypes.data_as(C.POINTER(C.c_float)), _stream()))
         return b.value, W
+
+    def selftest_wait_timeout(self):
+        self._ck(lib.nb_selftest_wait_timeout(self._h, _stream()))
 
     def check_guards(self):
         self._ck(lib.nb_check_guards(self._h, _stream()))

@@ -314,8 +314,8 @@ int nb_create(nb_ctx **out, int K, int64_t P, int M, float lr, float mom, int va
   if ((e = alloc_guarded(&c->X_base, &c->X, model_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(X)");
   if ((e = alloc_guarded(&c->V_base, &c->V, model_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(V)");
   if ((e = alloc_guarded(&c->acc_base, &c->acc, acc_bytes)) != cudaSuccess) return bail(e, "cudaMalloc(acc)");
-  if ((e = cudaMalloc(&c->d_err, sizeof(int))) != cudaSuccess) return bail(e, "cudaMalloc(err)");
-  if ((e = cudaMemset(c->d_err, 0, sizeof(int))) != cudaSuccess) return bail(e, "cudaMemset(err)");
+  if ((e = cudaMalloc(&c->d_err, 2 * sizeof(int))) != cudaSuccess) return bail(e, "cudaMalloc(err)");
+  if ((e = cudaMemset(c->d_err, 0, 2 * sizeof(int))) != cudaSuccess) return bail(e, "cudaMemset(err)");
   if (variant == NB_DPSGD || variant == NB_MATCHA) {
     if ((e = cudaMalloc(&c->d_mix, sizeof(nb::MixTable))) != cudaSuccess) return bail(e, "cudaMalloc(mix)");
     nb::MixTable *h = new (std::nothrow) nb::MixTable;
@@ -696,6 +696,26 @@ int nb_check_guards(nb_ctx *c, void *stream) {
                                          (q < kGuardBytes ? " before the array" : " after the array"));
   }
   return check_device_error(c, st);
+}
+
+int nb_selftest_wait_timeout(nb_ctx *c, void *stream) {
+  NB_ENTER(c);
+  cudaStream_t st = (cudaStream_t)stream;
+  int rc = check_device_error(c, st);  // start from a clean error word
+  if (rc != NB_OK) return rc;
+  int *gave_up = c->d_err + 1;
+  NB_CUDA(c, cudaMemsetAsync(gave_up, 0, sizeof(int), st));
+  NB_CUDA(c, nb::launch_wait_selftest(c->d_err, 9, 2000000ll /* ~1 ms */, gave_up, st));
+  c->launches++;
+  int h[2] = {0, 0};
+  NB_CUDA(c, cudaMemcpyAsync(h, c->d_err, 2 * sizeof(int), cudaMemcpyDeviceToHost, st));
+  NB_CUDA(c, cudaStreamSynchronize(st));
+  // the wait must have run out in every lane and reported its code; then the word is cleared again
+  NB_CUDA(c, cudaMemsetAsync(c->d_err, 0, 2 * sizeof(int), st));
+  NB_CUDA(c, cudaStreamSynchronize(st));
+  if (h[0] != 9 || h[1] != 32)
+    return fail(c, NB_ERR_STATE, "wait self-test: error word " + std::to_string(h[0]) + ", lanes that gave up " + std::to_string(h[1]));
+  return NB_OK;
 }
 
 int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan) {

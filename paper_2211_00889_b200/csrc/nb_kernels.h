@@ -60,6 +60,7 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan);
 cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, const PipePlan &plan, int *err_flag,
                                    cudaStream_t st);
 cudaError_t configure_pipeline();
+cudaError_t launch_wait_selftest(int *err_flag, int code, long long limit_cycles, int *gave_up, cudaStream_t st);
 cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan, int *err_flag, cudaStream_t st);
 
 // The same problem restricted to columns [c0, c0 + cols): every step of the path is independent per

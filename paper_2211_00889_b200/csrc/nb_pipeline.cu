@@ -77,14 +77,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the limit passes or another thread has already reported an
 // error; the caller then leaves its loop.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *err, int code) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *err, int code,
+                                          long long limit = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   int spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 63) == 0) {
       if (*reinterpret_cast<volatile int *>(err) != 0) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit) {
         atomicCAS(err, 0, code);
         return false;
       }
@@ -480,6 +481,20 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
   if (!ok) drain_and_exit_delay();
 }
 
+// Self-test of the bounded wait: one warp waits, with a short limit, on a barrier phase that nothing
+// will ever complete.  Every lane must give up, the error word must carry `code`, and the kernel
+// must return normally (no trap, the context stays usable).
+__global__ void nb_wait_selftest_kernel(int *err, int code, long long limit_cycles, int *gave_up) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(&bar, 0, err, code, limit_cycles);
+  if (!ok) atomicAdd(gave_up, 1);
+}
+
 struct PipeTuning {
   int enabled = 1, T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0;
   int sm_count = 0;
@@ -677,6 +692,11 @@ cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, 
     if (centralized) nb_stream_pipeline_kernel<4, kModeCentralized><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
     else nb_stream_pipeline_kernel<4, kModeAccumulate><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_wait_selftest(int *err_flag, int code, long long limit_cycles, int *gave_up, cudaStream_t st) {
+  nb_wait_selftest_kernel<<<1, 32, 0, st>>>(err_flag, code, limit_cycles, gave_up);
   return cudaGetLastError();
 }
 

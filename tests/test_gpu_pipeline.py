@@ -234,3 +234,26 @@ def test_in_place_and_out_of_place_steps_interleave(B):
     assert torch.equal(ref.get_mean_params(), mix.get_mean_params())
     mix.check_guards()
     ref.close(); mix.close()
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(B):
+    """The kernels' barrier waits are bounded.  The self-test makes one run out on purpose (a barrier
+    phase that nothing completes, limit ~1 ms): the lanes give up, the error word carries the code,
+    the kernel returns, and the context then steps normally."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 2 * 512, steps=2)
+    ctx = B.context_for(w)
+    orc = H.oracle_for(w, w.P)
+    x0 = WL.init_params(w)
+    ctx.set_params(torch.from_numpy(x0).cuda()); orc.set_params(x0)
+    ctx.selftest_wait_timeout()
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        payload, values = WL.gradients_np(w, t)
+        ctx.step_fused(H.to_device(payload), n)
+        orc.step(values, n.tolist())
+        if t == 0:
+            ctx.selftest_wait_timeout()                     # between steps as well
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+    ctx.check_guards()                                      # also reads the (cleared) device error word
+    ctx.close()
