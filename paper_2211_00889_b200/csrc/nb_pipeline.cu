@@ -605,6 +605,7 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
     if (slots >= 2 * groups) { found = true; break; }
   }
   if (!found) return false;
+  if ((a.P / T) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
   // When one item holds a learner's whole contribution (R >= M) two slots per group are enough to
   // keep the copies back to back, and deeper rings measured 1-4 % slower (MATCHA and all-reduce
   // workloads with M = 4); learners that need several items per tile use all the slots that fit.
@@ -638,6 +639,7 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   if (!encode_fn()) return false;
   const int T = 512;
   if (a.P < T) return false;
+  if ((a.P / T) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
   int R = es == 2 ? 8 : 4;
   if (R > a.M) R = a.M;
   int groups = centralized ? 1 : 2;
