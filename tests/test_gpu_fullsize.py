@@ -33,11 +33,23 @@ def _windows(P, rng, n_random=24, width=48):
     ("cfg5_scale_ring", 2),
 ])
 def test_full_size_sampled_columns(name, steps):
+    _full_size(WL.WORKLOADS[name], steps)
+
+
+def test_more_than_two_to_the_31_columns():
+    """Column indices beyond 32 bits: one learner pair, 2^31 + 1544 columns (the last window the
+    oracle checks lies entirely above 2^31)."""
+    from dataclasses import replace
+    w = replace(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], K=2, M=2, P=2 ** 31 + 3 * 512 + 8, name="two_to_31_columns")
+    _full_size(w, 2)
+
+
+def _full_size(w, steps):
     import torch
     from paper_2211_00889_b200.build import build_library
     build_library()
     from paper_2211_00889_b200 import binding as B
-    w = WL.WORKLOADS[name]
+    name = w.name
     es = 4 if w.grad_dtype == "f32" else 2
     need = w.K * w.M * w.P * es + 4 * w.K * w.P * 4 + w.M * w.P * 4 + (2 << 30)
     torch.cuda.empty_cache()
