@@ -11,8 +11,11 @@ device-side W builder runs first).  Prints ONE JSON line (rank 0).
   e2e       the same metric through nb_step_fused_host: pinned HOST gradient buffers, the H2D copies
             of the finished rows and the D2H copy of the mean model inside the timed region
   roofline  algorithmic bytes of one fused-step launch / its mean CUDA-event duration, against
-            the measured HBM copy bandwidth of this machine's B200s
-  cpu_baseline  the CPU oracle, as it stands, timed on a bounded column slice of the same workload
+            the measured HBM copy bandwidth of this machine's B200s; `sustained` repeats the same step
+            for at least two seconds and reports it against the clocks sampled meanwhile
+  workloads the other configurations, variants and entry points, one short run each (N = 1 only)
+  cpu_baseline  the CPU oracle, as it stands, timed on a bounded column slice of the same workload:
+            on one core and on every core the process may use (columns split over processes)
 
 With N > 1 (torchrun) every rank owns its own column shard of the same shape (weak scaling): the
 path is independent per column, so there is no data-path collective; ranks only meet in the
@@ -24,6 +27,7 @@ import os
 import sys
 import threading
 import time
+from dataclasses import replace
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
@@ -33,11 +37,14 @@ METRIC = "fused NB-SGD step throughput (params*learners/s)"
 UNIT = "params*learners/s"
 DEFAULT_WORKLOAD = "cfg3_dpsgd_ring_resnet50"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per algorithmic byte of the fused step kernel: dram__bytes_read.sum + dram__bytes_write.sum
-# of nb_step_pipeline_kernel over the algorithmic bytes of the same launch, from the ncu capture of an
-# 8M-column case of the default workload (summarised under profiles/).
-# Traffic grows in proportion to the columns a launch processes.
-TRAFFIC_PER_ALGORITHMIC_BYTE = 0.988
+
+# DRAM bytes per algorithmic byte, per (workload, entry): dram__bytes_read.sum + dram__bytes_write.sum
+# of the kernels of one step over the algorithmic bytes of the same step, from ncu captures of a
+# narrower column range of that workload (summarised under profiles/; traffic grows in proportion
+# to the columns).  No entry: no capture exists and `traffic` is reported as null.
+TRAFFIC_PER_ALGORITHMIC_BYTE = {
+    ("cfg3_dpsgd_ring_resnet50", "nb_step_fused"): 0.988,
+}
 
 
 def parse_args():
@@ -50,15 +57,24 @@ def parse_args():
     ap.add_argument("--variant", default="", choices=["", "allreduce", "dpsgd", "centralized"],
                     help="run the workload's sizes with another variant (dpsgd = ring)")
     ap.add_argument("--order", default="mix_then_update", choices=["mix_then_update", "update_then_mix"])
-    ap.add_argument("--unfused", action="store_true", help="time nb_accumulate + nb_step instead of nb_step_fused")
-    ap.add_argument("--grad-pad", type=int, default=0, help="experiment: extra elements of row pitch in the gradient buffers")
+    ap.add_argument("--entry", default="fused", choices=["fused", "unfused", "streaming"],
+                    help="fused: nb_step_fused; unfused: nb_accumulate + nb_step; streaming: one "
+                         "nb_accumulate_minibatch per finished mini-batch, then nb_step")
+    ap.add_argument("--unfused", action="store_true", help="same as --entry unfused")
     ap.add_argument("--cols", type=int, default=0, help="profiling aid: run the workload on this many columns instead of its P")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-cols", type=int, default=2_000_000)
-    ap.add_argument("--cpu-sample-steps", type=int, default=10)
-    return ap.parse_args()
+    ap.add_argument("--no-workloads", action="store_true", help="skip the table of other workloads / entries")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the >= 2 s repetition of the headline step")
+    ap.add_argument("--workload-steps", type=int, default=20, help="timed steps of every `workloads` entry")
+    ap.add_argument("--sustained-seconds", type=float, default=2.5)
+    ap.add_argument("--cpu-sample-cols", type=int, default=4_000_000)
+    ap.add_argument("--cpu-sample-steps", type=int, default=8)
+    a = ap.parse_args()
+    if a.unfused:
+        a.entry = "unfused"
+    return a
 
 
 def measured_peak():
@@ -77,12 +93,27 @@ def host_threads():
         return os.cpu_count() or 1
 
 
+ENTRY_NAMES = {"fused": "nb_step_fused", "unfused": "nb_accumulate+nb_step",
+               "streaming": "nb_accumulate_minibatch x sum(n_i) + nb_step"}
+
+
+def config_of(w, order, entry, world):
+    """Description of the timed workload; the same keys and values in both arms."""
+    es = 4 if w.grad_dtype == "f32" else 2
+    return {"workload": w.name, "K": w.K, "P": w.P, "M": w.M, "grad_dtype": w.grad_dtype, "variant": w.variant,
+            "topology": w.topology, "order": order, "entry": ENTRY_NAMES[entry],
+            "parallelism": "column-shard x%d" % world,
+            "l2": "inputs larger than L2 (%.1f GB gradient stream + %.1f GB state per step; no flush needed)"
+                  % (w.K * w.M * w.P * es / 1e9, 2 * w.K * w.P * 4 / 1e9)}
+
+
 # ---------------------------------------------------------------------------------------------
-# clocks: sampled through NVML while the timed region runs (read-only)
+# clocks: sampled through NVML while a timed region runs (read-only)
 # ---------------------------------------------------------------------------------------------
 class ClockSampler:
-    def __init__(self, index):
-        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+    def __init__(self, index, period=0.01):
+        self.index, self.samples, self.times, self.reasons, self.max_mhz = index, [], [], set(), None
+        self.period = period
         self._stop = threading.Event()
         self._thr = None
         try:
@@ -102,14 +133,16 @@ class ClockSampler:
                  "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4)}
         while not self._stop.is_set():
             try:
-                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                self.times.append(time.perf_counter())
+                self.samples.append(mhz)
                 r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
                 for k, bit in names.items():
                     if r & bit:
                         self.reasons.add(k)
             except Exception:
                 pass
-            time.sleep(0.01)
+            time.sleep(self.period)
 
     def start(self):
         if self.nv:
@@ -126,31 +159,35 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------------------------
-# CPU oracle timing (cpu_baseline leg and --impl reference)
+# CPU oracle timing (cpu_baseline legs and --impl reference)
 # ---------------------------------------------------------------------------------------------
-def time_oracle(w, sample_cols, steps, warmup=0):
-    """Times oracle.step on a column slice of workload w (exact: columns are independent).
-    Returns (params*learners/s, seconds per step, description)."""
+def _oracle_worker(job):
+    """Runs in a worker process (or inline): times oracle.step on columns [0, cols) of a workload
+    whose seed is offset per worker.  Returns the seconds of the timed steps, one per step."""
+    (wdict, cols, steps, warmup, worker) = job
+    for k in ("OMP_NUM_THREADS", "OPENBLAS_NUM_THREADS", "MKL_NUM_THREADS"):
+        os.environ[k] = "1"
     import numpy as np
     from oracle import nb_oracle as O
     from paper_2211_00889_b200 import workloads as WL
-    ws = WL.scaled(w, min(sample_cols, w.P))
+    w = WL.Workload(**wdict)
+    ws = replace(WL.scaled(w, cols), seed=w.seed + 7919 * worker)
     central = w.variant == "centralized"
     if w.variant in ("allreduce", "centralized"):
         orc = O.Oracle(ws.K, ws.P, ws.M, ws.lr, ws.mom, "allreduce")
     elif w.variant == "dpsgd":
         orc = O.Oracle(ws.K, ws.P, ws.M, ws.lr, ws.mom, "dpsgd", W=O.ring_W(ws.K))
     else:
-        partner = O.greedy_matchings(O.random_regular_graph(ws.seed, ws.K, ws.degree)[0], ws.K)
+        partner = O.greedy_matchings(O.random_regular_graph(w.seed, ws.K, ws.degree)[0], ws.K)
         orc = O.Oracle(ws.K, ws.P, ws.M, ws.lr, ws.mom, "matcha", partner=partner, alpha=ws.alpha,
-                       prob=ws.act_prob, seed=ws.seed)
+                       prob=ws.act_prob, seed=w.seed)
     x0 = WL.init_params(ws)
     orc.set_params(x0)
     x_ps, v_ps = x0.astype(np.float64), np.zeros(ws.P)
-    G = WL.gradients_torch(ws, 0, "cpu").float().numpy()     # one block, reused (not timed)
-    total = 0.0
+    G = WL.gradients_np(ws, 0)[1]                      # one block, reused (drawing it is not timed)
+    out = []
     for t in range(warmup + steps):
-        n = O.straggler_counts(ws.straggler_model, ws.seed, t, ws.K, ws.M, ws.straggler_params)
+        n = O.straggler_counts(w.straggler_model, w.seed, t, ws.K, ws.M, ws.straggler_params)
         t0 = time.perf_counter()
         if central:
             x_ps, v_ps = O.step_centralized(x_ps, v_ps, G, n, ws.lr, ws.mom)
@@ -158,25 +195,47 @@ def time_oracle(w, sample_cols, steps, warmup=0):
             orc.step(G, n)
         dt = time.perf_counter() - t0
         if t >= warmup:
-            total += dt
+            out.append((t0, t0 + dt))
+    return out
+
+
+def time_oracle(w, sample_cols, steps, warmup=0, procs=1):
+    """Times oracle.step on a column slice of workload w (exact: columns are independent), the
+    columns split evenly over `procs` worker processes, each running the oracle untouched on one
+    thread.  Returns (params*learners/s, seconds per step, description)."""
+    from dataclasses import asdict
+    cols = min(sample_cols, w.P)
+    per = max(1, cols // procs)
+    jobs = [(asdict(w), per, steps, warmup, r) for r in range(procs)]
+    if procs == 1:
+        spans = [_oracle_worker(jobs[0])]
+    else:
+        import multiprocessing as mp
+        with mp.get_context("spawn").Pool(procs) as pool:
+            spans = pool.map(_oracle_worker, jobs)
+    # Workers run concurrently but not in lock step: the sample's duration is the busiest worker's
+    # total over its timed steps (every worker does the same number of steps on the same width).
+    total = max(sum(b - a for a, b in s) for s in spans)
     per_step = total / steps
-    desc = "oracle.step (NumPy fp64, 1 thread) on a %d-column slice of %s, %d steps" % (ws.P, w.name, steps)
-    return ws.K * ws.P / per_step, per_step, desc
+    desc = ("oracle.step (NumPy fp64) on a %d-column slice of %s, %d steps, %d worker process%s of one thread each"
+            % (per * procs, w.name, steps, procs, "" if procs == 1 else "es (%d columns each)" % per))
+    return w.K * per * procs / per_step, per_step, desc
 
 
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    cols = max(1, args.cpu_sample_cols // 4)
-    value, per_step, desc = time_oracle(w, cols, args.steps, args.warmup)
+    cores = host_threads()
+    # a bounded sample per step: 125k columns per core keeps 25 steps within about a minute
+    cols = min(w.P, 125_000 * cores)
+    value, per_step, desc = time_oracle(w, cols, args.steps, args.warmup, procs=cores)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "K": w.K, "P": w.P, "M": w.M, "grad_dtype": w.grad_dtype,
-                   "variant": w.variant, "topology": w.topology},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "config": config_of(w, args.order, args.entry, max(1, args.gpus)),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -186,6 +245,202 @@ def run_reference(args, w):
 # ---------------------------------------------------------------------------------------------
 # the CUDA arm
 # ---------------------------------------------------------------------------------------------
+class Runner:
+    """One workload resident on the device: context, gradient buffers, and the timed loop."""
+
+    def __init__(self, B, WL, w, dev, order="mix_then_update", seed_offset=0, bufs=None, row_shift=0):
+        import torch
+        self.B, self.WL, self.w, self.dev, self.torch = B, WL, w, dev, torch
+        self.es = 4 if w.grad_dtype == "f32" else 2
+        g_bytes = w.K * w.M * w.P * self.es
+        wr = replace(w, seed=w.seed + seed_offset)
+        if bufs is None:
+            free, _ = torch.cuda.mem_get_info()
+            n_buf = 2 if free > 2 * g_bytes + 3 * w.K * w.P * 4 + (8 << 30) else 1
+            bufs = [WL.gradients_torch(wr, b, dev) for b in range(n_buf)]
+            if row_shift:      # the same stream `row_shift` elements off its allocation's 16-byte boundary
+                shifted = []
+                for b in bufs:
+                    flat = torch.empty(b.numel() + row_shift, dtype=b.dtype, device=dev)
+                    v = flat[row_shift:].view_as(b)
+                    v.copy_(b)
+                    shifted.append(v)
+                bufs = shifted
+        self.bufs = bufs
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(wr.seed)
+        x0 = torch.randn(w.P, generator=gen, device=dev, dtype=torch.float32) * w.init_sigma
+        self.ctx = B.context_for(w)
+        self.ctx.set_params(x0)
+        if order == "update_then_mix":
+            self.ctx.set_option(B.NB_OPT_ORDER, B.NB_ORDER_UPDATE_THEN_MIX)
+        self.order = order
+
+    def counts(self, t):
+        w = self.w
+        return self.B.straggler_sample(w.straggler_model, w.seed, t, w.K, w.M, w.straggler_params)[0]
+
+    def one_step(self, entry, g, n):
+        ctx = self.ctx
+        if entry == "fused":
+            ctx.step_fused(g, n)
+        elif entry == "unfused":
+            ctx.accumulate(g, n)
+            ctx.step()
+        else:
+            # Alg. 1 inner loop as the gradients arrive: round m delivers mini-batch m of every learner
+            # that finished it; the fastest learner's M-th delivery raises the terminal signal last
+            ctx.begin_iteration()
+            for m in range(self.w.M):
+                for i in range(self.w.K):
+                    if m < n[i]:
+                        ctx.accumulate_minibatch(i, g[i, m])
+            ctx.step()
+
+    def own_bytes(self, entry, n):
+        """Bytes the entry point itself must move in one step (its accumulator round trips included)."""
+        w, es = self.w, self.es
+        rows = 1 if w.variant == "centralized" else w.K
+        alg = w.P * (es * int(n.sum()) + 16 * rows)
+        if entry == "unfused":
+            return alg + 8 * w.K * w.P                                   # acc written once, read once
+        if entry == "streaming":                                           # acc read-modify-write per delivery
+            rmw = sum((2 * int(k) - 1) * 4 for k in n if k > 0) + 4 * w.K  # + the step's read of acc
+            return alg + w.P * rmw
+        return alg
+
+    def timed(self, entry, steps, warmup, t_first=0, sampler=None, barrier=None, per_step_events=True):
+        torch = self.torch
+        ctx, bufs = self.ctx, self.bufs
+        nb = len(bufs)
+        for t in range(t_first, t_first + warmup):
+            self.one_step(entry, bufs[t % nb], self.counts(t))
+        if barrier:
+            barrier()
+        else:
+            torch.cuda.synchronize()
+        launches0 = ctx.get_stats()["kernel_launches"]
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        alg, own, sum_n = [], 0.0, 0
+        if sampler:
+            sampler.start()
+        host_t0 = time.perf_counter()
+        e0.record()
+        for s in range(steps):
+            t = t_first + warmup + s
+            n = self.counts(t)                 # S0: host straggler simulator, inside the timed step
+            ev[s][0].record()
+            self.one_step(entry, bufs[t % nb], n)
+            ev[s][1].record()
+            st = ctx.get_stats()
+            alg.append(st["algorithmic_bytes"])
+            sum_n += st["sum_finished"]
+            own += self.own_bytes(entry, n)
+        e1.record()
+        if barrier:
+            barrier()
+        else:
+            torch.cuda.synchronize()
+        clocks = sampler.stop() if sampler else None
+        total_ms = e0.elapsed_time(e1)
+        step_ms = [a.elapsed_time(b) for a, b in ev]
+        launch_ms = sum(step_ms) / steps
+        return {"total_ms": total_ms, "launch_ms": launch_ms, "step_ms": step_ms, "alg_bytes": alg,
+                "own_bytes_per_step": own / steps, "mean_sum_finished": sum_n / steps,
+                "launches": ctx.get_stats()["kernel_launches"] - launches0, "clocks": clocks,
+                "kernel_plan": ctx.get_kernel_plan(), "host_t0": host_t0,
+                "step_start_ms": [e0.elapsed_time(a) for a, _ in ev]}
+
+    def close(self):
+        self.ctx.close()
+        self.bufs = None
+
+
+def table_entry(label, w, order, entry, r, peak, steps, note=None):
+    alg = sum(r["alg_bytes"]) / len(r["alg_bytes"])
+    ms = r["total_ms"] / steps
+    achieved = alg / (r["launch_ms"] * 1e-3) / 1e9
+    moved = r["own_bytes_per_step"] / (r["launch_ms"] * 1e-3) / 1e9
+    tr = TRAFFIC_PER_ALGORITHMIC_BYTE.get((w.name, ENTRY_NAMES[entry] if order == "mix_then_update"
+                                           else ENTRY_NAMES[entry] + "[update_then_mix]"))
+    out = {"name": label, "K": w.K, "P": w.P, "M": w.M, "grad_dtype": w.grad_dtype, "variant": w.variant,
+           "topology": w.topology, "order": order, "entry": ENTRY_NAMES[entry], "steps": steps,
+           "ms_per_step": ms, "step_ms_device": r["launch_ms"], "value": w.K * w.P / (ms * 1e-3), "unit": UNIT,
+           "algorithmic_bytes_per_step": alg, "achieved_hbm_gbs": achieved, "frac": achieved / peak,
+           "entry_bytes_per_step": r["own_bytes_per_step"], "entry_moved_gbs": moved, "entry_moved_frac": moved / peak,
+           "traffic": tr * alg if tr else None, "mean_sum_finished": r["mean_sum_finished"],
+           "gpu_launches_per_step": r["launches"] / steps, "kernel_plan": r["kernel_plan"], "clocks": r["clocks"]}
+    if note:
+        out["note"] = note
+    return out
+
+
+def sustained_leg(runner, seconds, est_ms, t_first, local):
+    """The headline step repeated back to back for at least `seconds`; GB/s against the SM clock
+    sampled meanwhile (a 1 kW part settles below its maximum clock under sw_power_cap)."""
+    steps = max(50, int(seconds * 1e3 / est_ms) + 1)
+    sampler = ClockSampler(local, period=0.02)
+    r = runner.timed("fused", steps, 3, t_first=t_first, sampler=sampler)
+    alg = r["alg_bytes"]
+    gbs = [a / (ms * 1e-3) / 1e9 for a, ms in zip(alg, r["step_ms"])]
+    total_alg = sum(alg)
+    ms_per_step = r["total_ms"] / steps
+    # clock of every step: the sample nearest to the step's start (device time since the region's
+    # first event, laid over the host clock at that event's record call)
+    times = [(t - r["host_t0"]) * 1e3 for t in sampler.times]
+    bins = {}
+    j = 0
+    for s, start in enumerate(r["step_start_ms"]):
+        while j + 1 < len(times) and abs(times[j + 1] - start) <= abs(times[j] - start):
+            j += 1
+        if times:
+            b = int(sampler.samples[j] // 100 * 100)
+            bins.setdefault(b, []).append(gbs[s])
+    med = lambda v: sorted(v)[len(v) // 2]
+    c = r["clocks"] or {}
+    return {"steps": steps, "seconds": r["total_ms"] * 1e-3, "ms_per_step": ms_per_step,
+            "achieved": total_alg / (sum(r["step_ms"]) * 1e-3) / 1e9, "unit": "GB/s",
+            "sm_mhz_median": c.get("sm_mhz"), "sm_max_mhz": c.get("sm_max_mhz"), "reasons": c.get("reasons"),
+            "clock_samples": c.get("samples"),
+            "ms_x_sm_mhz": (ms_per_step * c["sm_mhz"]) if c.get("sm_mhz") else None,
+            "gbs_by_sm_mhz_bin": {"%d-%d" % (b, b + 99): {"steps": len(v), "median_gbs": med(v)}
+                                  for b, v in sorted(bins.items())}}
+
+
+def other_workloads(args, B, WL, dev, base_runner, peak, local, log):
+    """One short run each of the other configurations, variants and entry points (N = 1)."""
+    import torch
+    out = []
+    steps, warm = args.workload_steps, 3
+    w3 = base_runner.w
+
+    def run(label, w, order="mix_then_update", entry="fused", bufs=None, row_shift=0, note=None):
+        t0 = time.time()
+        try:
+            r = Runner(B, WL, w, dev, order=order, bufs=bufs, row_shift=row_shift)
+            res = r.timed(entry, steps, warm, sampler=ClockSampler(local))
+            out.append(table_entry(label, w, order, entry, res, peak, steps, note))
+            r.close()
+            del r
+        except Exception as e:                      # a workload that cannot run is reported, not hidden
+            out.append({"name": label, "error": "%s: %s" % (type(e).__name__, e)})
+        torch.cuda.empty_cache()
+        log("%s: %.1f s" % (label, time.time() - t0))
+
+    # variants and entry points on the headline workload's own sizes and gradient buffers
+    shared = base_runner.bufs
+    run(w3.name + "[centralized]", replace(w3, variant="centralized", topology="full", name=w3.name + "[centralized]"),
+        bufs=shared, note="Alg. 3: one shared model, algorithmic bytes P*(e_g*sum n_i + 16)")
+    run(w3.name + "[update_then_mix]", w3, order="update_then_mix", bufs=shared, note="Eq. 4-6 order")
+    run(w3.name + "[unfused]", w3, entry="unfused", bufs=shared,
+        note="nb_accumulate + nb_step: the accumulator round trip (8*K*P bytes) is moved but not algorithmic")
+    run(w3.name + "[streaming]", w3, entry="streaming", bufs=shared,
+        note="Alg. 1 inner loop as the gradients arrive: one launch per finished mini-batch, accumulator "
+             "read-modify-write per delivery")
+    return out, shared
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -210,99 +465,63 @@ def run_ours(args, w):
         sharding.barrier()
         torch.cuda.synchronize()
 
+    def log(msg):
+        if rank == 0:
+            print("[bench] " + msg, file=sys.stderr, flush=True)
+
     # rank r owns columns [r*P, (r+1)*P) of an N*P-wide problem: same counts everywhere, own data
-    wr = WL.scaled(w, w.P)
-    from dataclasses import replace
-    wr = replace(wr, seed=w.seed + 1000 * rank)
-    es = 4 if w.grad_dtype == "f32" else 2
-    g_bytes = w.K * w.M * w.P * es
-    free, _ = torch.cuda.mem_get_info()
-    n_buf = 2 if free > 2 * g_bytes + 4 * w.K * w.P * 4 + (8 << 30) else 1
-    bufs = [WL.gradients_torch(wr, b, dev) for b in range(n_buf)]
-    ld = {}
-    if args.grad_pad:
-        wide = [torch.empty((w.K, w.M, w.P + args.grad_pad), dtype=b.dtype, device=dev) for b in bufs]
-        for dst, src in zip(wide, bufs):
-            dst[:, :, :w.P].copy_(src)
-        bufs = [b[:, :, :w.P] for b in wide]
-        ld = dict(ld_m=w.P + args.grad_pad, ld_k=w.M * (w.P + args.grad_pad))
-    gen = torch.Generator(device=dev)
-    gen.manual_seed(wr.seed)
-    x0 = torch.randn(w.P, generator=gen, device=dev, dtype=torch.float32) * w.init_sigma
-    ctx = B.context_for(w)
-    ctx.set_params(x0)
-    if args.order == "update_then_mix":
-        ctx.set_option(B.NB_OPT_ORDER, B.NB_ORDER_UPDATE_THEN_MIX)
-
-    def one_step(g, n):
-        if args.unfused:
-            ctx.accumulate(g, n, **ld)
-            ctx.step()
-        else:
-            ctx.step_fused(g, n, **ld)
-
-    def counts(t):
-        return B.straggler_sample(w.straggler_model, w.seed, t, w.K, w.M, w.straggler_params)[0]
-
-    total_steps = args.warmup + args.steps
-    for t in range(args.warmup):
-        one_step(bufs[t % n_buf], counts(t))
+    runner = Runner(B, WL, w, dev, order=args.order, seed_offset=1000 * rank)
+    es = runner.es
     if world > 1:   # every rank derives the counts by itself; they must coincide (checked outside the timed region)
-        assert sharding.counts_agree(counts(args.warmup), dev), "ranks disagree on the finished counts"
-    barrier()
-    launches0 = ctx.get_stats()["kernel_launches"]
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local)
-    alg_bytes = 0.0
-    sum_n = 0
-    sampler.start()
-    e0.record()
-    for s in range(args.steps):
-        t = args.warmup + s
-        n = counts(t)                      # S0: host straggler simulator, inside the timed step
-        ev[s][0].record()
-        one_step(bufs[t % n_buf], n)
-        ev[s][1].record()
-        st = ctx.get_stats()
-        alg_bytes += st["algorithmic_bytes"]
-        sum_n += st["sum_finished"]
-    e1.record()
-    barrier()
-    clocks = sampler.stop()
-    kernel_plan = ctx.get_kernel_plan()
-    launches = ctx.get_stats()["kernel_launches"] - launches0
-    total_ms = e0.elapsed_time(e1)
-    launch_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
-    total_ms_max = sharding.max_over_ranks(total_ms, dev)
+        assert sharding.counts_agree(runner.counts(args.warmup), dev), "ranks disagree on the finished counts"
+    r = runner.timed(args.entry, args.steps, args.warmup, sampler=ClockSampler(local), barrier=barrier)
+    total_ms_max = sharding.max_over_ranks(r["total_ms"], dev)
     ms_per_step = total_ms_max / args.steps
     value = w.K * w.P * world / (ms_per_step * 1e-3)
+    clocks, launches = r["clocks"], r["launches"]
 
     peak, peak_kind = measured_peak()
-    bytes_per_launch = alg_bytes / args.steps
-    achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
+    bytes_per_launch = sum(r["alg_bytes"]) / args.steps
+    achieved = bytes_per_launch / (r["launch_ms"] * 1e-3) / 1e9
+    tr = TRAFFIC_PER_ALGORITHMIC_BYTE.get((w.name.split("[")[0], ENTRY_NAMES[args.entry]
+                                           if args.order == "mix_then_update" and not args.variant else ""))
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_per_launch) if TRAFFIC_PER_ALGORITHMIC_BYTE else None,
-                "peak_source": "of " + peak_kind, "kernel": "nb_step_pipeline_kernel (fused accumulate+mix+momentum+update)",
-                "algorithmic_bytes_per_launch": bytes_per_launch, "launch_ms": launch_ms,
-                "frac_of_8TBps_nominal": achieved / 8000.0, "mean_sum_finished": sum_n / args.steps,
-                "kernel_plan": kernel_plan}
+                "traffic": tr * bytes_per_launch if tr else None,
+                "peak_source": "of " + peak_kind,
+                "kernel": "nb_step_pipeline_kernel (fused accumulate+mix+momentum+update)" if args.entry == "fused"
+                          else ENTRY_NAMES[args.entry],
+                "algorithmic_bytes_per_launch": bytes_per_launch, "launch_ms": r["launch_ms"],
+                "frac_of_8TBps_nominal": achieved / 8000.0, "mean_sum_finished": r["mean_sum_finished"],
+                "kernel_plan": r["kernel_plan"], "timed": "burst: the %d timed steps" % args.steps}
+    t_next = args.warmup + args.steps
+    single = rank == 0 and world == 1
+
+    if single and not args.no_sustained and args.entry == "fused":
+        roofline["sustained"] = sustained_leg(runner, args.sustained_seconds, r["launch_ms"], t_next, local)
+        roofline["sustained"]["frac"] = roofline["sustained"]["achieved"] / peak
+        log("sustained leg done")
+
+    workloads = None
+    if single and not args.no_workloads:
+        workloads, _ = other_workloads(args, B, WL, dev, runner, peak, local, log)
 
     # ---- end to end: host gradient buffers through nb_step_fused_host -------------------------
     e2e = None
     if not args.no_e2e:
+        ctx, bufs = runner.ctx, runner.bufs
         host = torch.empty((w.K, w.M, w.P), dtype=bufs[0].dtype, pin_memory=True)
         host.copy_(bufs[0])
         mean_out = torch.empty(w.P, dtype=torch.float32, pin_memory=True)
         torch.cuda.synchronize()
-        ctx.step_fused_host(host, counts(total_steps), mean_out=mean_out)   # warm-up: allocates staging
+        t_e2e = 1_000_000
+        ctx.step_fused_host(host, runner.counts(t_e2e), mean_out=mean_out)   # warm-up: allocates staging
         barrier()
         h2d = 0
         t0 = time.perf_counter()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record()
         for s in range(args.e2e_steps):
-            n = counts(total_steps + 1 + s)
+            n = runner.counts(t_e2e + 1 + s)
             ctx.step_fused_host(host, n, mean_out=mean_out)
             h2d += int(n.sum()) * w.P * es
         a1.record()
@@ -314,32 +533,79 @@ def run_ours(args, w):
                "steps": args.e2e_steps, "h2d_bytes_per_step": h2d // args.e2e_steps,
                "d2h_bytes_per_step": w.P * 4,
                "api": "nb_step_fused_host (pinned host gradients in, mean model out)"}
-        del host
+        del host, mean_out
+        log("e2e done")
+    runner.close()
+    del runner
+    torch.cuda.empty_cache()
+
+    if workloads is not None:
+        workloads += larger_workloads(args, B, WL, dev, w, peak, local, log)
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, per_step, desc = time_oracle(w, args.cpu_sample_cols, args.cpu_sample_steps)
-        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
-               "host_cores_available": host_threads()}
+    if single and not args.no_cpu_baseline:
+        cores = host_threads()
+        v1, _, d1 = time_oracle(w, args.cpu_sample_cols, args.cpu_sample_steps, procs=1)
+        log("cpu baseline, one core, done")
+        vn, _, dn = time_oracle(w, args.cpu_sample_cols, args.cpu_sample_steps, procs=cores)
+        cpu = {"value": vn, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": dn,
+               "one_core": {"value": v1, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": d1},
+               "host_cores_available": cores}
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "K": w.K, "P": w.P, "M": w.M, "grad_dtype": w.grad_dtype,
-                       "variant": w.variant, "topology": w.topology, "order": args.order,
-                       "entry": "nb_accumulate+nb_step" if args.unfused else "nb_step_fused",
-                       "parallelism": "column-shard x%d" % world,
-                       "l2": "inputs larger than L2 (%.1f GB gradient stream x%d buffers + %.1f GB state per step)"
-                             % (g_bytes / 1e9, n_buf, 2 * w.K * w.P * 4 / 1e9)},
+            "config": config_of(w, args.order, args.entry, world),
             "achieved_hbm_gbs": achieved, "frac_of_8TBps": achieved / 8000.0,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+            "workloads": workloads,
         }
         print(json.dumps(line), flush=True)
-    ctx.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def larger_workloads(args, B, WL, dev, w_head, peak, local, log):
+    """The configurations that need their own gradient streams, run after the headline's memory is free."""
+    import torch
+    out = []
+    steps, warm = args.workload_steps, 3
+
+    def run(label, w, order="mix_then_update", entry="fused", bufs=None, row_shift=0, note=None, keep=False):
+        t0 = time.time()
+        r = None
+        try:
+            r = Runner(B, WL, w, dev, order=order, bufs=bufs, row_shift=row_shift)
+            res = r.timed(entry, steps, warm, sampler=ClockSampler(local))
+            out.append(table_entry(label, w, order, entry, res, peak, steps, note))
+        except Exception as e:
+            out.append({"name": label, "error": "%s: %s" % (type(e).__name__, e)})
+        kept = r.bufs if (r is not None and keep) else None
+        if r is not None:
+            r.close()
+        del r
+        torch.cuda.empty_cache()
+        log("%s: %.1f s" % (label, time.time() - t0))
+        return kept
+
+    W = WL.WORKLOADS
+    # the headline workload with one more column: every gradient row starts at a different byte
+    # offset, none on a 16-byte boundary (per-row bulk copies instead of tensor-map boxes)
+    odd = replace(w_head, P=w_head.P + 1, name=w_head.name + "[P+1, rows not 16-byte aligned]")
+    run(odd.name, odd, note="dense odd row length: per-row bulk copies of the 16-byte aligned superset")
+    for name in ("cfg2_allreduce_resnet18", "cfg4_matcha_vgg16"):
+        if name != w_head.name:
+            run(name, W[name])
+    w5 = W["cfg5_scale_allreduce"]
+    kept = run(w5.name, w5, keep=True)
+    run("cfg5_scale_ring", W["cfg5_scale_ring"], bufs=kept)
+    del kept
+    torch.cuda.empty_cache()
+    k64 = replace(W["cfg3_dpsgd_ring_resnet50"], K=64, P=12_800_000, name="ring_K64_P12.8M")
+    run(k64.name, k64, note="the largest learner count the library takes (NB_MAX_K)")
+    return out
 
 
 def main():
@@ -347,10 +613,8 @@ def main():
     from paper_2211_00889_b200 import workloads as WL
     w = WL.WORKLOADS[args.workload]
     if args.cols:
-        from dataclasses import replace
         w = replace(WL.scaled(w, args.cols), name="%s[P=%d]" % (w.name, args.cols))
     if args.variant:
-        from dataclasses import replace
         topo = {"allreduce": "full", "dpsgd": "ring", "centralized": "full"}[args.variant]
         w = replace(w, variant=args.variant, topology=topo, name="%s[%s]" % (w.name, args.variant))
     if args.impl == "reference":

@@ -27,7 +27,15 @@
  *     retained; pointers marked "device" must stay valid until `stream` has passed the call's work;
  *   - a context is bound to the device that was current at nb_create and must be used from one host
  *     thread at a time;
- *   - a CUDA failure is reported as NB_ERR_CUDA and is sticky for that context.
+ *   - a CUDA failure is reported as NB_ERR_CUDA and is sticky for that context;
+ *   - the kernels' internal waits are bounded.  One that runs out (a defect, never seen in normal
+ *     operation) abandons the remaining tiles and records a code in a device word.  That word is
+ *     read only where the host already waits for the device: copies to host memory
+ *     (nb_get_params, nb_get_momentum, nb_get_accumulator, nb_get_mean_params with a host dst),
+ *     nb_step_fused_host and nb_check_guards, the explicit query.  It then becomes a sticky
+ *     NB_ERR_CUDA; models and momentum produced since the previous such point are invalid.  Calls
+ *     that only enqueue work (nb_accumulate, nb_step, nb_step_fused, outputs to device memory)
+ *     return NB_OK without looking at it.
  */
 #ifndef NB_H_
 #define NB_H_
@@ -59,7 +67,9 @@ enum nb_variant {
   NB_ALLREDUCE = 0,   /* W = (1/K) 1 1^T: mean over learners (Eq. 4-5)                              */
   NB_DPSGD = 1,       /* fixed sparse doubly-stochastic W (Eq. 6; Alg. 2)                           */
   NB_MATCHA = 2,      /* W(t) = I - alpha * sum of the Laplacians of the matchings active at t      */
-  NB_CENTRALIZED = 3  /* one parameter-server model shared by all learners (Alg. 3)                 */
+  NB_CENTRALIZED = 3  /* one parameter-server model shared by all learners (Alg. 3).  The server    */
+                      /* applies the MEAN of the learners' terms, (1/K) sum_i s_i acc_i (Eq. 2's    */
+                      /* 1/P), where Alg. 3 as printed sums them; pass lr * K to get the sum.        */
 };
 
 enum nb_dtype { NB_F32 = 0, NB_BF16 = 1 }; /* element type of the gradient stream */
@@ -93,8 +103,9 @@ typedef struct nb_topology {
 
 /* nb_set_option keys and values */
 enum nb_option {
-  NB_OPT_NORM = 0,  /* NB_NORM_MEAN (default) | NB_NORM_PAPER */
-  NB_OPT_ORDER = 1  /* NB_ORDER_MIX_THEN_UPDATE (default) | NB_ORDER_UPDATE_THEN_MIX */
+  NB_OPT_NORM = 0,   /* NB_NORM_MEAN (default) | NB_NORM_PAPER */
+  NB_OPT_ORDER = 1,  /* NB_ORDER_MIX_THEN_UPDATE (default) | NB_ORDER_UPDATE_THEN_MIX */
+  NB_OPT_KERNEL = 2  /* NB_KERNEL_AUTO (default) | NB_KERNEL_DIRECT */
 };
 enum nb_norm {
   NB_NORM_MEAN = 0,  /* s_i = 1/n_i: mean of the finished mini-batch gradients (s_i = 0 if n_i = 0)        */
@@ -103,6 +114,11 @@ enum nb_norm {
 enum nb_order {
   NB_ORDER_MIX_THEN_UPDATE = 0, /* Alg. 2: x_i <- sum_j W_ij x_j - lr v_i                                   */
   NB_ORDER_UPDATE_THEN_MIX = 1  /* Eq. 4-6: x_i <- sum_j W_ij (x_j - lr v_j)                                */
+};
+
+enum nb_kernel {
+  NB_KERNEL_AUTO = 0,   /* bulk-copy pipeline kernels wherever they apply, direct-load kernels elsewhere */
+  NB_KERNEL_DIRECT = 1  /* direct-load kernels only (same bits, slower): a cross-check for tests        */
 };
 
 /* ------------------------------------------------------------------------------------------------
@@ -202,22 +218,22 @@ const char *nb_last_error(const nb_ctx *c);
 int nb_set_option(nb_ctx *c, int key, int64_t value);
 int nb_set_lr(nb_ctx *c, float lr);
 
-/* Loads the models: per_learner = 0: x0[P] is given to every learner ("initialize local models
- * with the same initialization", Alg. 1); per_learner = 1: x0[K,P] dense.  x0: host or device.
+/* Loads the models: per_learner = 0: x0[P] is given to every learner (all learners start from
+ * one common model: initialisation line of Alg. 1); per_learner = 1: x0[K,P] dense.  x0: host or device.
  * Zeroes the momentum and the step counter.  NB_CENTRALIZED accepts only per_learner = 0. */
 int nb_set_params(nb_ctx *c, const float *x0, int per_learner, void *stream);
 
 /* Masked accumulate (step 1): acc[i,p] = sum_{m < finished[i]} grads[i,m,p], fp32 accumulation in
  * ascending m; rows m >= finished[i] are never read.
  * grads: device, element (i,m,p) at grads[i*ld_k + m*ld_m + p], dtype NB_F32 or NB_BF16;
- * ld_m, ld_k in elements, 0 = dense (ld_m = P, ld_k = M*P).  Alignment decides the kernel, never
- * the result (all paths give identical bits): with grads 16-byte aligned and ld_m, ld_k multiples of
- * 16 bytes the bulk-copy pipeline kernels cover all full 512-column tiles; with 4-element alignment
- * the direct kernels use 128-bit / 64-bit loads; anything else runs scalar loads, still on the GPU.
+ * ld_m, ld_k in elements, 0 = dense (ld_m = P, ld_k = M*P); grads must be aligned to its element
+ * size.  Alignment decides the kernel, never the result (all paths give identical bits): the
+ * bulk-copy pipeline kernels cover all full 512-column tiles of any stream - rows that are 16-byte
+ * aligned (grads, ld_m and ld_k multiples of 16 bytes) travel as tensor-map boxes, other rows as one
+ * bulk copy each of their 16-byte aligned superset (a few per cent slower; when grads itself is not
+ * 16-byte aligned the first tile goes to the direct kernels too); the direct kernels take the
+ * ragged tail with 128-bit / 64-bit loads where 4-element alignment allows and scalar loads elsewhere.
  * (Rows whose pitch is a multiple of 2 KB stream 1-2 % faster than other 16-byte multiples.)
- * With a sparse W, rows that are not 16-byte aligned are handled out of place: the first such
- * step allocates a second [K,P] model array (NB_ERR_NOMEM if that fails) and the two arrays trade
- * places after every such step; nothing changes for the caller.
  * finished: host [K], each in [0, M].  Errors: NB_ERR_ARG. */
 int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
                   const int32_t *finished, void *stream);
@@ -227,9 +243,10 @@ int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t
  * terminal signal.  nb_accumulate_minibatch adds grad[P] (device, NB_F32 or NB_BF16) to learner i's
  * accumulator in fp32 - the same sums, in the same order, as nb_accumulate - and counts it; when a
  * learner has delivered all M mini-batches it is the first finisher and the terminal signal is
- * raised ("Broadcast terminal signals if n = N"); every later call of the iteration returns
- * NB_ABANDONED (a status, not an error) without touching anything ("Break and abandon unfinished
- * mini-batches").  nb_step then runs on the counts collected.  nb_get_finished reports them. */
+ * raised (Alg. 1, inner loop: the learner whose count reaches N tells the others); every later
+ * call of the iteration returns NB_ABANDONED (a status, not an error) without touching anything
+ * (Alg. 1: the other learners leave their loop and drop what they have not finished).  nb_step
+ * then runs on the counts collected.  nb_get_finished reports them. */
 #define NB_ABANDONED 1
 int nb_begin_iteration(nb_ctx *c);
 int nb_accumulate_minibatch(nb_ctx *c, int learner, const void *grad, int dtype, void *stream);
@@ -295,11 +312,13 @@ int nb_check_guards(nb_ctx *c, void *stream);
  * about a second; when one runs out the context reports a sticky NB_ERR_CUDA.) */
 int nb_selftest_wait_timeout(nb_ctx *c, void *stream);
 
-/* Which kernel shape ran the most recent step (for reports and tests), host out plan[8]:
+/* Which kernel shape ran the most recent step (for reports and tests), host out plan[10]:
  * [0] 1 if the bulk-copy pipeline kernel covered the full tiles, 0 if the direct-load kernel did
  * everything; [1] tile width in columns; [2] consumer groups per CTA; [3] ring slots per CTA;
  * [4] gradient rows per ring item; [5] CTAs launched; [6] dynamic shared memory per CTA in bytes;
- * [7] tiles covered (columns beyond [7]*[1] went to the direct-load kernel). */
+ * [7] tiles covered; [8] 0 if the gradient rows travelled as tensor-map boxes, 1 if as one bulk
+ * copy per row (rows not 16-byte aligned); [9] columns before the first covered tile (they, and the
+ * columns after [9] + [7]*[1], went to the direct-load kernel). */
 int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan);
 
 /* ------------------------------------------------------------------------------------------------
@@ -312,8 +331,10 @@ int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan);
  * order) entirely on memory the caller passes in, plus ONE piece of scratch: the fp32 accumulator
  * between the accumulate kernel and the update kernel, which is a fixed array inside the library
  * image of NB_STATIC_MAX_ELEMS floats (16 MiB; every GPU that loads the library holds it until the
- * process exits).  No context is needed and nothing is allocated or freed, by the CUDA runtime or
- * by any library, in any call.
+ * process exits).  No context is needed, and no call after the first on a device allocates or
+ * frees anything, through the CUDA runtime or any library (the first call resolves the array's
+ * address, which is also when a lazily loading driver brings the library's code and this array onto
+ * the device).
  *
  *   X, V      device, in/out, [K, ld] fp32 models and momentum, 16-byte aligned, ld >= P and a
  *             multiple of 4; columns [P, ld) of each row are padding the call may overwrite
@@ -323,7 +344,8 @@ int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan);
  *   - K*ld must not exceed NB_STATIC_MAX_ELEMS: larger problems are rejected with
  *     NB_ERR_UNSUPPORTED and a message (nb_last_error(NULL)); nothing is launched.
  *   - The first call on each device resolves the array's device address (once, with that device
- *     current); make that first call during set-up, before any stream capture is begun.
+ *     current); make that first call during set-up, before any stream capture is begun.  The
+ *     address is cached per device ordinal and is stale after cudaDeviceReset.
  *   - All calls on a device share the one array.  A call overwrites every element it later reads,
  *     so no state leaks from one call to the next, but two calls whose kernels overlap on the GPU
  *     (different streams, different threads, different contexts of the library) race on it:

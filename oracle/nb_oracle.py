@@ -187,8 +187,8 @@ def finished_mask(n, M):
 # Topologies and mixing matrices
 # ----------------------------------------------------------------------------------------------
 def full_W(K):
-    """All-reduce variant: W = (1/K) 1 1^T (Eq. 5 written as a mixing matrix)."""
-    return np.full((K, K), f32(1.0 / K), dtype=np.float64)
+    """All-reduce variant: W = (1/K) 1 1^T (Eq. 5 written as a mixing matrix), with the exact 1/K."""
+    return np.full((K, K), 1.0 / K, dtype=np.float64)
 
 
 def ring_W(K):

@@ -16,7 +16,8 @@ NB_OK, NB_ERR_ARG, NB_ERR_STATE, NB_ERR_CUDA, NB_ERR_NOMEM, NB_ERR_UNSUPPORTED =
 NB_ALLREDUCE, NB_DPSGD, NB_MATCHA, NB_CENTRALIZED = 0, 1, 2, 3
 NB_F32, NB_BF16 = 0, 1
 NB_TOPO_FULL, NB_TOPO_RING, NB_TOPO_CSR, NB_TOPO_MATCHINGS, NB_TOPO_RANDOM_REGULAR = 0, 1, 2, 3, 4
-NB_OPT_NORM, NB_OPT_ORDER = 0, 1
+NB_OPT_NORM, NB_OPT_ORDER, NB_OPT_KERNEL = 0, 1, 2
+NB_KERNEL_AUTO, NB_KERNEL_DIRECT = 0, 1
 NB_NORM_MEAN, NB_NORM_PAPER = 0, 1
 NB_ORDER_MIX_THEN_UPDATE, NB_ORDER_UPDATE_THEN_MIX = 0, 1
 NB_STRAG_UNIFORM_COUNT, NB_STRAG_SHIFTED_EXP, NB_STRAG_SHIFTED_EXP_SLOWSET = 0, 1, 2
@@ -279,8 +280,22 @@ class NbContext:
     def _finished(n):
         return np.ascontiguousarray(n, dtype=np.int32)
 
+    @staticmethod
+    def _pitches(grads, ld_m, ld_k):
+        """Element strides of a [K, M, P] gradient tensor: the caller's, else the tensor's own (a view
+        whose rows are contiguous is passed as it is, never copied)."""
+        if hasattr(grads, "stride") and grads.dim() == 3:
+            if grads.stride(2) != 1 and grads.shape[2] > 1:
+                raise ValueError("gradient rows must be contiguous (stride 1 along the parameter axis)")
+            if not ld_m:
+                ld_m = grads.stride(1) if grads.shape[1] > 1 else 0
+            if not ld_k:
+                ld_k = grads.stride(0) if grads.shape[0] > 1 else 0
+        return ld_m, ld_k
+
     def accumulate(self, grads, finished, ld_m=0, ld_k=0):
         n = self._finished(finished)
+        ld_m, ld_k = self._pitches(grads, ld_m, ld_k)
         self._ck(lib.nb_accumulate(self._h, _ptr(grads), _dtype_code(grads), ld_m, ld_k, _i32p(n), _stream()))
 
     def begin_iteration(self):
@@ -305,10 +320,12 @@ class NbContext:
 
     def step_fused(self, grads, finished, ld_m=0, ld_k=0):
         n = self._finished(finished)
+        ld_m, ld_k = self._pitches(grads, ld_m, ld_k)
         self._ck(lib.nb_step_fused(self._h, _ptr(grads), _dtype_code(grads), ld_m, ld_k, _i32p(n), _stream()))
 
     def step_fused_host(self, grads_host, finished, mean_out=None, ld_m=0, ld_k=0):
         n = self._finished(finished)
+        ld_m, ld_k = self._pitches(grads_host, ld_m, ld_k)
         self._ck(lib.nb_step_fused_host(self._h, _ptr(grads_host), _dtype_code(grads_host), ld_m, ld_k, _i32p(n),
                                         _ptr(mean_out), _stream()))
 
@@ -368,9 +385,10 @@ class NbContext:
         self._ck(lib.nb_check_guards(self._h, _stream()))
 
     def get_kernel_plan(self):
-        a = np.zeros(8, dtype=np.int32)
+        a = np.zeros(10, dtype=np.int32)
         self._ck(lib.nb_get_kernel_plan(self._h, _i32p(a)))
-        keys = ("pipeline", "tile", "groups", "slots", "rows_per_item", "grid", "smem_bytes", "tiles")
+        keys = ("pipeline", "tile", "groups", "slots", "rows_per_item", "grid", "smem_bytes", "tiles", "row_copies",
+                "head")
         return dict(zip(keys, (int(v) for v in a)))
 
     def get_stats(self):

@@ -16,16 +16,12 @@ struct nb_ctx {
   int K = 0, M = 0, rows = 0;  // rows = model rows held (K, or 1 for NB_CENTRALIZED)
   int64_t P = 0, ldx = 0;
   float lr = 0.f, mom = 0.f;
-  int variant = NB_ALLREDUCE, norm = NB_NORM_MEAN, order = NB_ORDER_MIX_THEN_UPDATE;
+  int variant = NB_ALLREDUCE, norm = NB_NORM_MEAN, order = NB_ORDER_MIX_THEN_UPDATE, kernel = NB_KERNEL_AUTO;
   nb::Mixing mx;
   float *X = nullptr, *V = nullptr, *acc = nullptr, *d_mean = nullptr;
   // X, V and acc sit between guard bands (kGuardBytes of a fixed byte pattern before and after);
   // nb_check_guards verifies that no kernel wrote outside its arrays.
   unsigned char *X_base = nullptr, *V_base = nullptr, *acc_base = nullptr;
-  // second model array for the out-of-place step (allocated the first time that kernel is needed);
-  // after such a step X and X2 trade places
-  float *X2 = nullptr;
-  unsigned char *X2_base = nullptr;
   size_t model_bytes = 0, acc_bytes = 0;
   nb::MixTable *d_mix = nullptr;
   int32_t *d_partner = nullptr;
@@ -129,13 +125,12 @@ int fill_step_args(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_
   const int es = dtype == NB_F32 ? 4 : 2;
   if (ld_m == 0) ld_m = c->P;
   if (ld_k == 0) ld_k = (int64_t)c->M * ld_m;
+  if ((uintptr_t)grads % (size_t)es != 0) return fail(c, NB_ERR_ARG, "grads is not aligned to its element size");
   if (ld_m < c->P) return fail(c, NB_ERR_ARG, "ld_m is smaller than P");
   if (ld_k < (int64_t)(c->M - 1) * ld_m + c->P) return fail(c, NB_ERR_ARG, "ld_k is too small for M rows of pitch ld_m");
-  int64_t sum = 0;
   for (int i = 0; i < c->K; ++i) {
     if (finished[i] < 0 || finished[i] > c->M)
       return fail(c, NB_ERR_ARG, "finished[" + std::to_string(i) + "] is outside [0, M]");
-    sum += finished[i];
   }
   std::memset(a, 0, sizeof(*a));
   a->X = c->X;
@@ -152,7 +147,6 @@ int fill_step_args(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_
   a->g_aligned = ((uintptr_t)grads % (size_t)(4 * es) == 0) && (ld_m % 4 == 0) && (ld_k % 4 == 0);
   for (int i = 0; i < c->K; ++i) a->n[i] = finished[i];
   *esize = es;
-  (void)sum;
   return NB_OK;
 }
 
@@ -200,29 +194,12 @@ int build_device_mixing(nb_ctx *c, cudaStream_t st) {
 
 // The step kernels on the columns `a` describes (all of them, or one chunk); the mixing matrix of
 // the current step must already be on the device.
-int launch_update(nb_ctx *c, const nb::StepArgs &a, int src, cudaStream_t st, bool whole_range = false) {
+int launch_update(nb_ctx *c, const nb::StepArgs &a, int src, cudaStream_t st) {
   int n_launched = 0;
+  const bool pipeline = c->kernel == NB_KERNEL_AUTO;
   cudaError_t e;
-  if (c->variant == NB_CENTRALIZED) {
-    e = nb::launch_centralized(a, src, c->d_err, &n_launched, st);
-  } else if (whole_range && nb::prefers_out_of_place(a, src)) {
-    // rows the bulk-copy kernel cannot take: read the old models from X, write the new ones to X2, swap
-    if (!c->X2) {
-      cudaError_t ea = alloc_guarded(&c->X2_base, &c->X2, c->model_bytes);
-      if (ea != cudaSuccess) return cuda_fail(c, ea, "cudaMalloc(X2)");
-    }
-    nb::StepArgs b = a;
-    b.X_out = c->X2;
-    e = nb::launch_step_out_of_place(b, src, st);
-    n_launched = 1;
-    c->last_plan = nb::PipePlan{};
-    if (e == cudaSuccess) {
-      std::swap(c->X, c->X2);
-      std::swap(c->X_base, c->X2_base);
-    }
-  } else {
-    e = nb::launch_step(a, src, c->d_err, &n_launched, &c->last_plan, st);
-  }
+  if (c->variant == NB_CENTRALIZED) e = nb::launch_centralized(a, src, pipeline, c->d_err, &n_launched, st);
+  else e = nb::launch_step(a, src, pipeline, c->d_err, &n_launched, &c->last_plan, st);
   c->launches += n_launched;
   if (e != cudaSuccess) return cuda_fail(c, e, "launch_step");
   return NB_OK;
@@ -232,7 +209,7 @@ int run_update(nb_ctx *c, nb::StepArgs *a, int src, cudaStream_t st) {
   fill_update_args(c, a);
   int rc = build_device_mixing(c, st);
   if (rc != NB_OK) return rc;
-  rc = launch_update(c, *a, src, st, true);
+  rc = launch_update(c, *a, src, st);
   if (rc != NB_OK) return rc;
   c->step++;
   c->acc_fresh = false;
@@ -345,7 +322,6 @@ int nb_destroy(nb_ctx *c) {
   DeviceGuard guard(c->device);
   cudaDeviceSynchronize();
   cudaFree(c->X_base);
-  cudaFree(c->X2_base);
   cudaFree(c->V_base);
   cudaFree(c->acc_base);
   cudaFree(c->d_mean);
@@ -375,6 +351,11 @@ int nb_set_option(nb_ctx *c, int key, int64_t value) {
   if (key == NB_OPT_ORDER) {
     if (value != NB_ORDER_MIX_THEN_UPDATE && value != NB_ORDER_UPDATE_THEN_MIX) return fail(c, NB_ERR_ARG, "unknown order");
     c->order = (int)value;
+    return NB_OK;
+  }
+  if (key == NB_OPT_KERNEL) {
+    if (value != NB_KERNEL_AUTO && value != NB_KERNEL_DIRECT) return fail(c, NB_ERR_ARG, "unknown kernel choice");
+    c->kernel = (int)value;
     return NB_OK;
   }
   return fail(c, NB_ERR_ARG, "unknown option key");
@@ -415,8 +396,8 @@ int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t
   int rc = fill_step_args(c, grads, dtype, ld_m, ld_k, finished, &a, &es);
   if (rc != NB_OK) return rc;
   int n_launched = 0;
-  cudaError_t e = nb::launch_accumulate(a, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16, c->d_err, &n_launched,
-                                        (cudaStream_t)stream);
+  cudaError_t e = nb::launch_accumulate(a, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16, c->kernel == NB_KERNEL_AUTO,
+                                        c->d_err, &n_launched, (cudaStream_t)stream);
   c->launches += n_launched;
   if (e != cudaSuccess) return cuda_fail(c, e, "launch_accumulate");
   std::memcpy(c->n_acc, a.n, sizeof(c->n_acc));
@@ -506,7 +487,9 @@ int nb_step_fused_host(nb_ctx *c, const void *grads_host, int dtype, int64_t ld_
   const size_t es = dtype == NB_F32 ? 4 : 2;
   if (ld_m == 0) ld_m = c->P;
   if (ld_k == 0) ld_k = (int64_t)c->M * ld_m;
+  if ((uintptr_t)grads_host % es != 0) return fail(c, NB_ERR_ARG, "grads_host is not aligned to its element size");
   if (ld_m < c->P) return fail(c, NB_ERR_ARG, "ld_m is smaller than P");
+  if (ld_k < (int64_t)(c->M - 1) * ld_m + c->P) return fail(c, NB_ERR_ARG, "ld_k is too small for M rows of pitch ld_m");
   for (int i = 0; i < c->K; ++i)
     if (finished[i] < 0 || finished[i] > c->M) return fail(c, NB_ERR_ARG, "finished count outside [0, M]");
   const int64_t ldg = (c->P + 511) / 512 * 512;  // staging pitch, elements: rows start on 2 KB boundaries
@@ -681,8 +664,7 @@ int nb_check_guards(nb_ctx *c, void *stream) {
   cudaStream_t st = (cudaStream_t)stream;
   unsigned char h[2 * kGuardBytes];
   struct Arr { const char *name; unsigned char *base; size_t bytes; };
-  const Arr arrs[4] = {{"X", c->X_base, c->model_bytes}, {"V", c->V_base, c->model_bytes}, {"acc", c->acc_base, c->acc_bytes},
-                       {"X (second array)", c->X2_base, c->model_bytes}};
+  const Arr arrs[3] = {{"X", c->X_base, c->model_bytes}, {"V", c->V_base, c->model_bytes}, {"acc", c->acc_base, c->acc_bytes}};
   for (const Arr &a : arrs) {
     if (!a.base) continue;
     NB_CUDA(c, cudaMemcpyAsync(h, a.base, kGuardBytes, cudaMemcpyDeviceToHost, st));
@@ -729,6 +711,8 @@ int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan) {
   plan[5] = p.grid;
   plan[6] = p.smem_bytes;
   plan[7] = p.n_tiles;
+  plan[8] = p.row_copies;
+  plan[9] = p.head;
   return NB_OK;
 }
 

@@ -161,55 +161,6 @@ __global__ void __launch_bounds__(256) nb_step_kernel(const __grid_constant__ St
 }
 
 // -------------------------------------------------------------------------------------------------
-// Out-of-place form of the sparse-W step in the Alg. 2 order: x_i(new) = sum_j W_ij x_j(old) - lr v_i
-// with the old models read straight from X (the neighbours' tiles hit in L1/L2: the same CTA touches
-// them within a few microseconds) and the new ones written to X_out.  No staging, hence no shared
-// memory beyond the W table and full occupancy.  Used when the bulk-copy kernel cannot take the
-// stream (rows that are not 16-byte aligned).  Same operation sequence as nb_step_kernel.
-// -------------------------------------------------------------------------------------------------
-template <int SRC, bool ALIGNED>
-__global__ void __launch_bounds__(256) nb_step_out_of_place_kernel(const __grid_constant__ StepArgs a) {
-  extern __shared__ float4 smem[];
-  const int tid = threadIdx.x, tpb = blockDim.x, K = a.K;
-  int32_t *s_col = reinterpret_cast<int32_t *>(smem);
-  float *s_val = reinterpret_cast<float *>(s_col + a.mix_slots);
-  int32_t *s_beg = reinterpret_cast<int32_t *>(s_val + a.mix_slots);
-  int32_t *s_end = s_beg + K;
-  for (int e = tid; e < a.mix_slots; e += tpb) {
-    s_col[e] = a.mix->col[e];
-    s_val[e] = a.mix->val[e];
-  }
-  for (int e = tid; e < K; e += tpb) {
-    s_beg[e] = a.mix->row_beg[e];
-    s_end[e] = a.mix->row_end[e];
-  }
-  __syncthreads();
-  const int64_t col0 = ((int64_t)blockIdx.x * tpb + tid) * kColsPerThread;
-  if (col0 >= a.P) return;
-  const int nvalid = (a.P - col0 < 4) ? (int)(a.P - col0) : 4;
-  const float *Xin = a.X + col0;
-  float *Xout = a.X_out + col0;
-  float *Vc = a.V + col0;
-  const int64_t ldx = a.ldx;
-  for (int i = 0; i < K; ++i) {
-    const float4 v = ld4(Vc + (int64_t)i * ldx);
-    const float4 g = gather<SRC, ALIGNED>(a, i, col0, nvalid);
-    const float4 vn = momentum(a.mom, v, a.s[i], g);
-    float4 xh = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int e = s_beg[i]; e < s_end[i]; ++e) {
-      const float w = s_val[e];
-      const float4 x = __ldg(reinterpret_cast<const float4 *>(Xin + (int64_t)s_col[e] * ldx));
-      xh.x = __fmaf_rn(w, x.x, xh.x);
-      xh.y = __fmaf_rn(w, x.y, xh.y);
-      xh.z = __fmaf_rn(w, x.z, xh.z);
-      xh.w = __fmaf_rn(w, x.w, xh.w);
-    }
-    st4(Vc + (int64_t)i * ldx, vn);
-    st4(Xout + (int64_t)i * ldx, descend(xh, a.lr, vn));
-  }
-}
-
-// -------------------------------------------------------------------------------------------------
 // Non-blocking synchronous centralized step (Alg. 3): one shared model.
 //   g = (1/K) sum_i s_i acc_i ; v <- mom v + g ; x <- x - lr v
 // -------------------------------------------------------------------------------------------------
@@ -315,9 +266,6 @@ cudaError_t configure_kernels() {
 }
 
 namespace {
-// Column range [done, P) of the same problem: what the direct-load kernels take over after a
-// pipeline kernel has covered the full tiles.
-StepArgs tail_of(const StepArgs &a, int64_t done, int es) { return column_range(a, done, a.P - done, es); }
 // The accumulator presented as a one-row fp32 gradient stream (0 + acc == acc bit for bit: acc is never -0).
 StepArgs acc_as_stream(const StepArgs &a) {
   StepArgs p = a;
@@ -340,31 +288,9 @@ StepArgs column_range(const StepArgs &a, int64_t c0, int64_t cols, int es) {
   return r;
 }
 
-cudaError_t launch_accumulate(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st) {
-  *launches = 0;
-  const int es = src == kSrcBF16 ? 2 : 4;
-  PipePlan plan;
-  int64_t done = 0;
-  if (plan_stream(a, es, false, &plan)) {
-    // cudaErrorNotSupported: the driver refused a tensor map for this memory (nothing was launched);
-    // the direct-load kernel then takes the whole range
-    cudaError_t e = launch_stream_pipeline(a, es, false, plan, err_flag, st);
-    if (e == cudaSuccess) {
-      ++*launches;
-      done = (int64_t)plan.n_tiles * plan.T;
-    } else if (e != cudaErrorNotSupported) {
-      return e;
-    }
-  }
-  if (done < a.P) {
-    cudaError_t e = launch_accumulate_direct_only(tail_of(a, done, es), src, st);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-  }
-  return cudaSuccess;
-}
+namespace {
 
-cudaError_t launch_accumulate_direct_only(const StepArgs &a, int src, cudaStream_t st) {
+cudaError_t launch_accumulate_direct(const StepArgs &a, int src, cudaStream_t st) {
   const int tpb = 256;
   const int64_t per_block = (int64_t)tpb * kColsPerThread;
   dim3 grid((unsigned)((a.P + per_block - 1) / per_block), (unsigned)a.K);
@@ -378,62 +304,101 @@ cudaError_t launch_accumulate_direct_only(const StepArgs &a, int src, cudaStream
   return cudaGetLastError();
 }
 
-namespace {
-StepArgs acc_as_stream(const StepArgs &a);
-}
-static cudaError_t launch_step_direct(const StepArgs &a, int src, cudaStream_t st) {
+cudaError_t launch_step_direct(const StepArgs &a, int src, cudaStream_t st) {
   if (src == kSrcAcc) return launch_step_t<kSrcAcc, true>(a, st);
   if (src == kSrcF32) return a.g_aligned ? launch_step_t<kSrcF32, true>(a, st) : launch_step_t<kSrcF32, false>(a, st);
   return a.g_aligned ? launch_step_t<kSrcBF16, true>(a, st) : launch_step_t<kSrcBF16, false>(a, st);
 }
 
-cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st) { return launch_step_direct(a, src, st); }
-
-bool prefers_out_of_place(const StepArgs &a, int src) {
-  if (a.mean_mode || a.order != NB_ORDER_MIX_THEN_UPDATE) return false;
-  const int es = src == kSrcBF16 ? 2 : 4;
-  const StepArgs p = src == kSrcAcc ? acc_as_stream(a) : a;
-  PipePlan plan;
-  return !plan_pipeline(p, es, &plan);
-}
-
-cudaError_t launch_step_out_of_place(const StepArgs &a, int src, cudaStream_t st) {
+cudaError_t launch_centralized_direct(const StepArgs &a, int src, cudaStream_t st) {
   const int tpb = 256;
   const int64_t per_block = (int64_t)tpb * kColsPerThread;
   const unsigned grid = (unsigned)((a.P + per_block - 1) / per_block);
-  const size_t smem = (size_t)a.mix_slots * 8 + (size_t)a.K * 8;
-#define NB_OOP(SRC, AL) nb_step_out_of_place_kernel<SRC, AL><<<grid, tpb, smem, st>>>(a)
-  if (src == kSrcAcc) NB_OOP(kSrcAcc, true);
-  else if (src == kSrcF32) { if (a.g_aligned) NB_OOP(kSrcF32, true); else NB_OOP(kSrcF32, false); }
-  else { if (a.g_aligned) NB_OOP(kSrcBF16, true); else NB_OOP(kSrcBF16, false); }
-#undef NB_OOP
+  if (src == kSrcAcc) nb_centralized_kernel<kSrcAcc, true><<<grid, tpb, 0, st>>>(a);
+  else if (src == kSrcF32) {
+    if (a.g_aligned) nb_centralized_kernel<kSrcF32, true><<<grid, tpb, 0, st>>>(a);
+    else nb_centralized_kernel<kSrcF32, false><<<grid, tpb, 0, st>>>(a);
+  } else {
+    if (a.g_aligned) nb_centralized_kernel<kSrcBF16, true><<<grid, tpb, 0, st>>>(a);
+    else nb_centralized_kernel<kSrcBF16, false><<<grid, tpb, 0, st>>>(a);
+  }
   return cudaGetLastError();
 }
 
-cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, PipePlan *used, cudaStream_t st) {
+// Covers all P columns of `a`: the bulk-copy kernel on the tiles `plan` names (when there is a plan),
+// the direct-load kernel on the columns before and after them.  `p` is `a` as the bulk-copy kernel
+// sees it (the unfused step presents the accumulator as a one-row gradient stream).
+// pipe(range, plan) returns cudaErrorNotSupported when the driver refused a tensor map for this
+// memory: nothing was launched then, and the direct-load kernel takes the whole range.
+template <typename Pipe, typename Direct>
+cudaError_t cover_columns(const StepArgs &a, const StepArgs &p, int es, const PipePlan *plan, int *launches,
+                          PipePlan *used, Pipe pipe, Direct direct) {
   *launches = 0;
-  *used = PipePlan{};
-  // The pipeline kernel sees one gradient-like stream; the unfused step presents the accumulator as one.
-  const int es = src == kSrcBF16 ? 2 : 4;
-  const StepArgs p = src == kSrcAcc ? acc_as_stream(a) : a;
-  PipePlan plan;
-  int64_t done = 0;
-  if (plan_pipeline(p, es, &plan)) {
-    cudaError_t e = launch_step_pipeline(p, es, plan, err_flag, st);
+  if (used) *used = PipePlan{};
+  int64_t lo = 0, hi = 0;  // columns [lo, hi) are done by the bulk-copy kernel
+  if (plan) {
+    const int64_t c0 = plan->head, cols = (int64_t)plan->n_tiles * plan->T;
+    cudaError_t e = pipe(column_range(p, c0, cols, es), *plan);
     if (e == cudaSuccess) {
       ++*launches;
-      *used = plan;
-      done = (int64_t)plan.n_tiles * plan.T;
-    } else if (e != cudaErrorNotSupported) {  // NotSupported: no tensor map for this memory, nothing launched
+      if (used) *used = *plan;
+      lo = c0;
+      hi = c0 + cols;
+    } else if (e != cudaErrorNotSupported) {
       return e;
     }
   }
-  if (done < a.P) {  // ragged tail (or everything, when the pipeline does not apply)
-    cudaError_t e = launch_step_direct(tail_of(a, done, es), src, st);
+  if (lo > 0) {  // the first tile of a stream that does not start on a 16-byte boundary
+    cudaError_t e = direct(column_range(a, 0, lo, es));
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  if (hi < a.P) {  // ragged tail (or everything, when the bulk-copy kernel does not apply)
+    cudaError_t e = direct(column_range(a, hi, a.P - hi, es));
     if (e != cudaSuccess) return e;
     ++*launches;
   }
   return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_accumulate_direct_only(const StepArgs &a, int src, cudaStream_t st) {
+  return launch_accumulate_direct(a, src, st);
+}
+cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st) { return launch_step_direct(a, src, st); }
+
+cudaError_t launch_accumulate(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, cudaStream_t st) {
+  const int es = src == kSrcBF16 ? 2 : 4;
+  PipePlan plan;
+  const bool planned = pipeline && plan_stream(a, es, false, &plan);
+  return cover_columns(
+      a, a, es, planned ? &plan : nullptr, launches, nullptr,
+      [&](const StepArgs &r, const PipePlan &pl) { return launch_stream_pipeline(r, es, false, pl, err_flag, st); },
+      [&](const StepArgs &r) { return launch_accumulate_direct(r, src, st); });
+}
+
+cudaError_t launch_step(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, PipePlan *used,
+                        cudaStream_t st) {
+  const int es = src == kSrcBF16 ? 2 : 4;
+  const StepArgs p = src == kSrcAcc ? acc_as_stream(a) : a;
+  PipePlan plan;
+  const bool planned = pipeline && plan_pipeline(p, es, &plan);
+  return cover_columns(
+      a, p, es, planned ? &plan : nullptr, launches, used,
+      [&](const StepArgs &r, const PipePlan &pl) { return launch_step_pipeline(r, es, pl, err_flag, st); },
+      [&](const StepArgs &r) { return launch_step_direct(r, src, st); });
+}
+
+cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, cudaStream_t st) {
+  const int es = src == kSrcBF16 ? 2 : 4;
+  const StepArgs p = src == kSrcAcc ? acc_as_stream(a) : a;
+  PipePlan plan;
+  const bool planned = pipeline && plan_stream(p, es, true, &plan);
+  return cover_columns(
+      a, p, es, planned ? &plan : nullptr, launches, nullptr,
+      [&](const StepArgs &r, const PipePlan &pl) { return launch_stream_pipeline(r, es, true, pl, err_flag, st); },
+      [&](const StepArgs &r) { return launch_centralized_direct(r, src, st); });
 }
 
 cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,
@@ -445,46 +410,6 @@ cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool al
   } else {
     if (aligned) nb_add_minibatch_kernel<kSrcBF16, true><<<grid, 256, 0, st>>>(acc_row, g, P, first);
     else nb_add_minibatch_kernel<kSrcBF16, false><<<grid, 256, 0, st>>>(acc_row, g, P, first);
-  }
-  return cudaGetLastError();
-}
-
-static cudaError_t launch_centralized_direct(const StepArgs &a, int src, cudaStream_t st);
-
-cudaError_t launch_centralized(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st) {
-  *launches = 0;
-  const int es = src == kSrcBF16 ? 2 : 4;
-  const StepArgs p = src == kSrcAcc ? acc_as_stream(a) : a;
-  PipePlan plan;
-  int64_t done = 0;
-  if (plan_stream(p, es, true, &plan)) {
-    cudaError_t e = launch_stream_pipeline(p, es, true, plan, err_flag, st);
-    if (e == cudaSuccess) {
-      ++*launches;
-      done = (int64_t)plan.n_tiles * plan.T;
-    } else if (e != cudaErrorNotSupported) {
-      return e;
-    }
-  }
-  if (done < a.P) {
-    cudaError_t e = launch_centralized_direct(tail_of(a, done, es), src, st);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-  }
-  return cudaSuccess;
-}
-
-static cudaError_t launch_centralized_direct(const StepArgs &a, int src, cudaStream_t st) {
-  const int tpb = 256;
-  const int64_t per_block = (int64_t)tpb * kColsPerThread;
-  const unsigned grid = (unsigned)((a.P + per_block - 1) / per_block);
-  if (src == kSrcAcc) nb_centralized_kernel<kSrcAcc, true><<<grid, tpb, 0, st>>>(a);
-  else if (src == kSrcF32) {
-    if (a.g_aligned) nb_centralized_kernel<kSrcF32, true><<<grid, tpb, 0, st>>>(a);
-    else nb_centralized_kernel<kSrcF32, false><<<grid, tpb, 0, st>>>(a);
-  } else {
-    if (a.g_aligned) nb_centralized_kernel<kSrcBF16, true><<<grid, tpb, 0, st>>>(a);
-    else nb_centralized_kernel<kSrcBF16, false><<<grid, tpb, 0, st>>>(a);
   }
   return cudaGetLastError();
 }

@@ -25,7 +25,6 @@ enum GradSource : int { kSrcF32 = 0, kSrcBF16 = 1, kSrcAcc = 2 };
 // Everything one step needs, passed by value as a kernel parameter (no per-step uploads).
 struct StepArgs {
   float *X;            // [K, ldx] models (NB_CENTRALIZED: [1, ldx])
-  float *X_out;        // out-of-place kernel only: where the new models go (never aliases X)
   float *V;            // [K, ldx] momentum
   float *acc;          // [K, ldx] accumulator (written by accumulate, read by the unfused step)
   const void *G;       // gradient stream, element (i,m,p) at G[i*ld_k + m*ld_m + p]
@@ -54,6 +53,8 @@ struct MatchaArgs {
 // Bulk-copy pipeline kernel (nb_pipeline.cu)
 struct PipePlan {
   int T, rows_per_item, n_slots, n_groups, smem_bytes, n_tiles, grid;  // all 0: the pipeline kernel did not run
+  int head;        // columns [0, head) left to the direct-load kernel (a stream whose start is not 16-byte aligned)
+  int row_copies;  // 0: gradient rows travel as tensor-map boxes; 1: one bulk copy per row (rows not 16-byte aligned)
 };
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan);
 bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan);
@@ -69,22 +70,17 @@ StepArgs column_range(const StepArgs &a, int64_t c0, int64_t cols, int es);
 
 int step_threads_per_block(const StepArgs &a);
 // Masked accumulate on all P columns (pipeline kernel on the full tiles when it applies).
-cudaError_t launch_accumulate(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st);
+cudaError_t launch_accumulate(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, cudaStream_t st);
 cudaError_t launch_accumulate_direct_only(const StepArgs &a, int src, cudaStream_t st);
-// Runs the step on all P columns: pipeline kernel on the full tiles when it applies, direct-load
-// kernel on the rest.  *launches receives the number of kernels launched.
-cudaError_t launch_step(const StepArgs &a, int src, int *err_flag, int *launches, PipePlan *used, cudaStream_t st);
-// True when launch_step would run the whole range on the direct-load kernel with a sparse W in the
-// Alg. 2 order: then an out-of-place step (models read from X, written to a second array) avoids the
-// shared-memory staging that limits that kernel's occupancy.
-bool prefers_out_of_place(const StepArgs &a, int src);
-// The out-of-place step on all P columns: reads a.X, writes a.X_out (caller swaps the two afterwards).
-cudaError_t launch_step_out_of_place(const StepArgs &a, int src, cudaStream_t st);
+// Runs the step on all P columns: pipeline kernel on the full tiles when it applies (and `pipeline`
+// allows it), direct-load kernel on the rest.  *launches receives the number of kernels launched.
+cudaError_t launch_step(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, PipePlan *used,
+                        cudaStream_t st);
 // The direct-load step kernel on all P columns (no pipeline kernel, no device error word).
 cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st);
 cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,
                                  cudaStream_t st);
-cudaError_t launch_centralized(const StepArgs &a, int src, int *err_flag, int *launches, cudaStream_t st);
+cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, cudaStream_t st);
 cudaError_t launch_matcha_build(const MatchaArgs &a, cudaStream_t st);
 cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, cudaStream_t st);
 cudaError_t configure_kernels();

@@ -25,6 +25,14 @@
 //     sequence as the direct-load kernels (bit-identical results), stores x_i and v_i with 128-bit
 //     stores and hands the slot back through its "empty" barrier.
 //
+// Gradient rows whose byte addresses are not multiples of 16 (odd row lengths, a stream that starts
+// at an odd element) cannot be described by a tensor map.  They take the same path with one change
+// (template parameter GA = false): the producer WARP issues one plain 1-D bulk copy per finished row,
+// lane r for row m0 + r, that fetches the 16-byte aligned superset of the row's tile segment (start
+// rounded down, T*ES + 16 bytes), and the consumers read each row at its own byte shift from shared
+// memory, element by element.  The momentum and model rows are library-owned, 2 KB-pitched and keep
+// their box copies.  Same additions in the same order: identical bits.
+//
 // No CTA ever waits on another CTA.  Every mbarrier wait is bounded: after ~1 s of cycles a
 // waiting thread records an error code in global memory, all roles drain and the kernel returns
 // (the host reports it as an error status); nothing traps.
@@ -109,6 +117,13 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, i
       "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
       : "memory");
 }
+// Plain 1-D bulk copy global -> shared: both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
 __device__ __forceinline__ void drain_and_exit_delay() {
   const long long t0 = clock64();
   while (clock64() - t0 < kDrainCycles) {
@@ -127,45 +142,94 @@ struct PipeArgs {
   int32_t n_tiles;        // full tiles covered by the kernel
   int32_t n_groups;       // consumer groups (each T/4 threads)
   int *err;               // device word: 0, or the code of the wait that ran out
+  // GA = false only: the gradient stream as bytes; (address & 15) of G and of the two pitches
+  const unsigned char *g_base;
+  int64_t g_ld_m_bytes, g_ld_k_bytes;
+  int32_t g_mis0, g_mis_m, g_mis_k;
   alignas(64) CUtensorMap xmap;                   // X as [K, units]: box = (256, K)
   alignas(64) CUtensorMap vmap;                   // V as [K, units]: box = (256, 1)
   alignas(64) CUtensorMap gmap[kMaxRowsPerItem];  // G as [K, M, units]: box = (256, r, 1), r = 1..R
 };
 
+// Four consecutive columns of one staged gradient row, widened to fp32.  GA: p is 16-byte (fp32) or
+// 8-byte (bf16) aligned; otherwise p is only element-aligned and the elements are read one by one.
+template <int SRC, bool GA>
+__device__ __forceinline__ float4 ld_row4(const unsigned char *p) {
+  if constexpr (GA) {
+    Raw<SRC> raw;
+    if constexpr (SRC == kSrcBF16) raw.r = *reinterpret_cast<const uint2 *>(p);
+    else raw.r = *reinterpret_cast<const float4 *>(p);
+    return widen(raw);
+  } else if constexpr (SRC == kSrcBF16) {
+    const uint16_t *e = reinterpret_cast<const uint16_t *>(p);
+    return make_float4(__uint_as_float((uint32_t)e[0] << 16), __uint_as_float((uint32_t)e[1] << 16),
+                       __uint_as_float((uint32_t)e[2] << 16), __uint_as_float((uint32_t)e[3] << 16));
+  } else {
+    const float *e = reinterpret_cast<const float *>(p);
+    return make_float4(e[0], e[1], e[2], e[3]);
+  }
+}
+
 // acc += row_0 + row_1 + ... (ascending, one add at a time) over N rows `stride` bytes apart; all
 // loads are issued before the first add.  Same sequence of fp32 additions as a plain loop.
-template <int SRC, int N>
-__device__ __forceinline__ float4 sum_rows_n(float4 acc, const unsigned char *rowp, int stride) {
-  Raw<SRC> raw[N];
+// GA = false: row r sits at its own byte shift (s0 + r * mis_m) & 15 inside its staged superset.
+template <int SRC, bool GA, int N>
+__device__ __forceinline__ float4 sum_rows_n(float4 acc, const unsigned char *rowp, int stride, int s0, int mis_m) {
+  float4 g[N];
 #pragma unroll
   for (int r = 0; r < N; ++r) {
-    if constexpr (SRC == kSrcBF16) raw[r].r = *reinterpret_cast<const uint2 *>(rowp + r * stride);
-    else raw[r].r = *reinterpret_cast<const float4 *>(rowp + r * stride);
+    const int shift = GA ? 0 : ((s0 + r * mis_m) & 15);
+    g[r] = ld_row4<SRC, GA>(rowp + r * stride + shift);
   }
 #pragma unroll
-  for (int r = 0; r < N; ++r) acc = add4(acc, widen(raw[r]));
+  for (int r = 0; r < N; ++r) acc = add4(acc, g[r]);
   return acc;
 }
-template <int SRC>
-__device__ __forceinline__ float4 sum_rows(float4 acc, const unsigned char *rowp, int stride, int rows) {
+template <int SRC, bool GA>
+__device__ __forceinline__ float4 sum_rows(float4 acc, const unsigned char *rowp, int stride, int rows, int s0,
+                                           int mis_m) {
   switch (rows) {
     case 0: return acc;
-    case 1: return sum_rows_n<SRC, 1>(acc, rowp, stride);
-    case 2: return sum_rows_n<SRC, 2>(acc, rowp, stride);
-    case 3: return sum_rows_n<SRC, 3>(acc, rowp, stride);
-    case 4: return sum_rows_n<SRC, 4>(acc, rowp, stride);
-    case 5: return sum_rows_n<SRC, 5>(acc, rowp, stride);
-    case 6: return sum_rows_n<SRC, 6>(acc, rowp, stride);
-    case 7: return sum_rows_n<SRC, 7>(acc, rowp, stride);
-    default: return sum_rows_n<SRC, 8>(acc, rowp, stride);
+    case 1: return sum_rows_n<SRC, GA, 1>(acc, rowp, stride, s0, mis_m);
+    case 2: return sum_rows_n<SRC, GA, 2>(acc, rowp, stride, s0, mis_m);
+    case 3: return sum_rows_n<SRC, GA, 3>(acc, rowp, stride, s0, mis_m);
+    case 4: return sum_rows_n<SRC, GA, 4>(acc, rowp, stride, s0, mis_m);
+    case 5: return sum_rows_n<SRC, GA, 5>(acc, rowp, stride, s0, mis_m);
+    case 6: return sum_rows_n<SRC, GA, 6>(acc, rowp, stride, s0, mis_m);
+    case 7: return sum_rows_n<SRC, GA, 7>(acc, rowp, stride, s0, mis_m);
+    default: return sum_rows_n<SRC, GA, 8>(acc, rowp, stride, s0, mis_m);
   }
+}
+
+// Producer side of one ring item's gradient rows.  GA: lane 0 issues one box of exactly `rows` rows.
+// Otherwise lanes 0..rows-1 each fetch the aligned superset of one row's tile segment.
+template <int ES, bool GA>
+__device__ __forceinline__ void issue_rows(const PipeArgs &a, unsigned char *dst, int T, int tile, int i, int m0,
+                                           int rows, int lane, uint64_t *bar) {
+  if constexpr (GA) {
+    if (rows > 0) tma_load_3d(dst, &a.gmap[rows - 1], tile * kBoxInner, m0, i, bar);
+  } else {
+    if (lane < rows) {
+      const unsigned char *src = a.g_base + (int64_t)i * a.g_ld_k_bytes + (int64_t)(m0 + lane) * a.g_ld_m_bytes +
+                                 (int64_t)tile * (T * ES);
+      src -= reinterpret_cast<uintptr_t>(src) & 15;
+      bulk_load_1d(dst + lane * (T * ES + 16), src, (uint32_t)(T * ES + 16), bar);
+    }
+  }
+}
+
+// Bytes of one ring slot: the momentum row (step kernel only) followed by R staged gradient rows,
+// rounded up to 128 bytes, the alignment a tiled bulk copy needs for its shared-memory destination.
+__host__ __device__ inline int slot_bytes_of(int v_bytes, int T, int es, int R, int row_pad) {
+  return (v_bytes + R * (T * es + row_pad) + 127) / 128 * 128;
 }
 
 struct PipeLayout {
   int32_t off_tab, off_xs, off_slots, slot_bytes, total;
 };
 
-__host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, int n_slots, int mix_slots) {
+// row_pad: 0 for box copies, 16 when every row is staged as its 16-byte aligned superset.
+__host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, int n_slots, int mix_slots, int row_pad) {
   PipeLayout L;
   int off = (2 * n_slots + 5) * 8;
   off = (off + 127) / 128 * 128;
@@ -175,21 +239,23 @@ __host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, i
   L.off_xs = off;
   off += 2 * K * T * 4;  // the X stage is double-buffered: tile t+1's models load while tile t is consumed
   L.off_slots = off;
-  L.slot_bytes = T * 4 + R * T * es;
+  L.slot_bytes = slot_bytes_of(T * 4, T, es, R, row_pad);
   L.total = off + n_slots * L.slot_bytes;
   return L;
 }
 
 // ES = bytes per gradient element (2: bf16, 4: fp32).
 // TT = tile width known at compile time (512, the usual shape: strides become immediates) or 0 (a.T).
-template <int ES, bool MEAN, int TT>
+// GA = gradient rows are 16-byte aligned (box copies through tensor maps) or not (one bulk copy per row).
+template <int ES, bool MEAN, int TT, bool GA>
 __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeline_kernel(const __grid_constant__ PipeArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
+  constexpr int kRowPad = GA ? 0 : 16;
   const StepArgs &s = a.s;
   const int K = s.K, T = TT ? TT : a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
   const int NSG = NS / NG;  // slots in each group's ring
-  const PipeLayout L = pipe_layout(K, T, ES, R, NS, s.mix_slots);
+  const PipeLayout L = pipe_layout(K, T, ES, R, NS, s.mix_slots, kRowPad);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);
   uint64_t *empty = full + NS;
   uint64_t *xfull = empty + NS;
@@ -233,28 +299,31 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
   bool ok = true;
 
   if (warp < NG) {
-    // ------------------------------------------- item producers: one thread per consumer group
-    // Producer g (lane 0 of warp g) feeds group g's private ring with the items of the learners
-    // i = g, g+NG, ... ; a slot is always filled for, and released by, the same group, in order,
-    // which is what makes waiting on a phase parity unambiguous, and a slow group never holds up
-    // the copies of another.
-    if (lane == 0) {
+    // ------------------------------------------- item producers: one per consumer group
+    // Producer g (warp g; lane 0 alone when the rows travel as boxes) feeds group g's private ring
+    // with the items of the learners i = g, g+NG, ... ; a slot is always filled for, and released
+    // by, the same group, in order, which is what makes waiting on a phase parity unambiguous, and
+    // a slow group never holds up the copies of another.
+    if (!GA || lane == 0) {
       const int g = warp;
       uint32_t slot = 0, phase = 0;
       for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x) {
-        const int c0 = tile * kBoxInner;  // the tile's first unit in every map
         for (int i = g; ok && i < K; i += NG) {
           const int n = s.n[i];
           int m0 = 0;
           do {
             const int rows = (n - m0 < R) ? (n - m0) : R;
             const uint32_t sl = (uint32_t)g * NSG + slot;
-            if (!(ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2))) break;
+            if constexpr (GA) ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2);
+            else ok = __all_sync(0xffffffffu, mbar_wait(&empty[sl], phase ^ 1, a.err, 2));
+            if (!ok) break;
             unsigned char *dst = slots + (size_t)sl * L.slot_bytes;
-            const uint32_t bytes = (uint32_t)(rows * T * ES + (m0 == 0 ? T * 4 : 0));
-            mbar_expect_tx(&full[sl], bytes);
-            if (m0 == 0) tma_load_2d(dst, &a.vmap, c0, i, &full[sl]);
-            if (rows > 0) tma_load_3d(dst + T * 4, &a.gmap[rows - 1], c0, m0, i, &full[sl]);
+            if (lane == 0) {
+              mbar_expect_tx(&full[sl], (uint32_t)(rows * (T * ES + kRowPad) + (m0 == 0 ? T * 4 : 0)));
+              if (m0 == 0) tma_load_2d(dst, &a.vmap, tile * kBoxInner, i, &full[sl]);
+            }
+            if constexpr (!GA) __syncwarp();
+            issue_rows<ES, GA>(a, dst + T * 4, T, tile, i, m0, rows, lane, &full[sl]);
             if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
             m0 += R;
           } while (m0 < n);
@@ -312,7 +381,8 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
             if (!ok) break;
             const unsigned char *src = slots + (size_t)sl * L.slot_bytes;
             if (m0 == 0) v = reinterpret_cast<const float4 *>(src)[cq];
-            acc = sum_rows<SRC>(acc, src + T * 4 + cq * 4 * ES, T * ES, rows);
+            const int s0 = GA ? 0 : (a.g_mis0 + i * a.g_mis_k + m0 * a.g_mis_m);
+            acc = sum_rows<SRC, GA>(acc, src + T * 4 + cq * 4 * ES, T * ES + kRowPad, rows, s0, a.g_mis_m);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[sl]);
             if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
@@ -371,24 +441,25 @@ constexpr int kModeAccumulate = 0, kModeCentralized = 1;
 struct StreamLayout {
   int32_t off_slots, slot_bytes, total;
 };
-__host__ __device__ inline StreamLayout stream_layout(int T, int es, int R, int n_slots) {
+__host__ __device__ inline StreamLayout stream_layout(int T, int es, int R, int n_slots, int row_pad) {
   StreamLayout L;
   int off = 2 * n_slots * 8;
   off = (off + 127) / 128 * 128;
   L.off_slots = off;
-  L.slot_bytes = R * T * es;
+  L.slot_bytes = slot_bytes_of(0, T, es, R, row_pad);
   L.total = off + n_slots * L.slot_bytes;
   return L;
 }
 
-template <int ES, int MODE>
+template <int ES, int MODE, bool GA>
 __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline_kernel(const __grid_constant__ PipeArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
+  constexpr int kRowPad = GA ? 0 : 16;
   const StepArgs &s = a.s;
   const int K = s.K, T = a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
   const int NSG = NS / NG;
-  const StreamLayout L = stream_layout(T, ES, R, NS);
+  const StreamLayout L = stream_layout(T, ES, R, NS, kRowPad);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);
   uint64_t *empty = full + NS;
   unsigned char *slots = smem_raw + L.off_slots;
@@ -406,20 +477,22 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
   bool ok = true;
 
   if (warp < NG) {
-    if (lane == 0) {  // producer of group `warp`
+    if (!GA || lane == 0) {  // producer of group `warp`
       const int g = warp;
       uint32_t slot = 0, phase = 0;
       for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x) {
-        const int c0 = tile * kBoxInner;
         for (int i = g; ok && i < K; i += NG) {
           const int n = s.n[i];
           int m0 = 0;
           do {
             const int rows = (n - m0 < R) ? (n - m0) : R;
             const uint32_t sl = (uint32_t)g * NSG + slot;
-            if (!(ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2))) break;
-            mbar_expect_tx(&full[sl], (uint32_t)(rows * T * ES));  // 0 rows: a plain arrival
-            if (rows > 0) tma_load_3d(slots + (size_t)sl * L.slot_bytes, &a.gmap[rows - 1], c0, m0, i, &full[sl]);
+            if constexpr (GA) ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2);
+            else ok = __all_sync(0xffffffffu, mbar_wait(&empty[sl], phase ^ 1, a.err, 2));
+            if (!ok) break;
+            if (lane == 0) mbar_expect_tx(&full[sl], (uint32_t)(rows * (T * ES + kRowPad)));  // 0 rows: a plain arrival
+            if constexpr (!GA) __syncwarp();
+            issue_rows<ES, GA>(a, slots + (size_t)sl * L.slot_bytes, T, tile, i, m0, rows, lane, &full[sl]);
             if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
             m0 += R;
           } while (m0 < n);
@@ -448,11 +521,10 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
           ok = __all_sync(0xffffffffu, mbar_wait(&full[sl], phase, a.err, 4));
           if (!ok) break;
           const unsigned char *rowp = slots + (size_t)sl * L.slot_bytes + (size_t)cq * 4 * ES;
+          const int s0 = GA ? 0 : (a.g_mis0 + i * a.g_mis_k + m0 * a.g_mis_m);
           for (int r = 0; r < rows; ++r) {
-            Raw<SRC> raw;
-            if constexpr (ES == 2) raw.r = *reinterpret_cast<const uint2 *>(rowp + (size_t)r * T * ES);
-            else raw.r = *reinterpret_cast<const float4 *>(rowp + (size_t)r * T * ES);
-            acc = add4(acc, widen(raw));
+            const int shift = GA ? 0 : ((s0 + r * a.g_mis_m) & 15);
+            acc = add4(acc, ld_row4<SRC, GA>(rowp + (size_t)r * (T * ES + kRowPad) + shift));
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&empty[sl]);
@@ -496,25 +568,34 @@ __global__ void nb_wait_selftest_kernel(int *err, int code, long long limit_cycl
 }
 
 struct PipeTuning {
-  int enabled = 1, T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0;
+  int T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0;
   int sm_count = 0;
 };
 
+// Shape overrides for tuning sweeps.  Only a library built with -DNB_TUNING reads them (from the
+// environment, once per process); the shipped build always takes the planner's own choice.
 PipeTuning &tuning() {
   static PipeTuning t = [] {
     PipeTuning q;
+#ifdef NB_TUNING
     auto geti = [](const char *name, int dflt) {
       const char *v = std::getenv(name);
       return v ? std::atoi(v) : dflt;
     };
-    q.enabled = geti("NB_PIPELINE", 1);
     q.T = geti("NB_PIPELINE_TILE", 0);
     q.slots = geti("NB_PIPELINE_SLOTS", 0);
     q.ctas_per_sm = geti("NB_PIPELINE_CTAS_PER_SM", 0);
     q.rows = geti("NB_PIPELINE_ROWS", 0);
     q.groups = geti("NB_PIPELINE_GROUPS", 0);
+#endif
     return q;
   }();
+  if (t.sm_count == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&t.sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (t.sm_count <= 0) t.sm_count = 148;
+  }
   return t;
 }
 
@@ -557,6 +638,40 @@ bool encode_map(CUtensorMap *map, const void *base, int unit_bytes, int rank, co
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Which columns the bulk-copy kernels may cover, given how the gradient stream is aligned.
+//   16-byte aligned rows: box copies, tiles [0, P / T).
+//   otherwise: one bulk copy per row of the 16-byte aligned superset of its tile segment, which reads
+//   up to 15 bytes before the segment and up to 16 bytes after it.  Both stay inside the caller's
+//   stream if (a) the first tile is left out when G itself is not 16-byte aligned (`head` columns go
+//   to the direct-load kernel) and (b) the last tile covered ends at least 16 bytes before the end of
+//   a row.
+struct Coverage {
+  bool rows_aligned;
+  int64_t head;     // columns [0, head) are left to the direct-load kernel
+  int64_t n_tiles;  // tiles covered, starting at column `head`
+};
+Coverage coverage(const StepArgs &a, int es, int T) {
+  Coverage c;
+  c.rows_aligned = (uintptr_t)a.G % 16 == 0 && (a.ld_m * es) % 16 == 0 && (a.ld_k * es) % 16 == 0;
+  if (c.rows_aligned) {
+    c.head = 0;
+    c.n_tiles = a.P / T;
+  } else {
+    c.head = (uintptr_t)a.G % 16 == 0 ? 0 : T;
+    c.n_tiles = (a.P - c.head - 16 / es) / T;
+    if (a.P - c.head - 16 / es < 0) c.n_tiles = 0;
+  }
+  return c;
+}
+
+void fill_row_args(PipeArgs *p, const StepArgs &a, int es) {
+  p->g_base = reinterpret_cast<const unsigned char *>(a.G);
+  p->g_ld_m_bytes = a.ld_m * es;
+  p->g_ld_k_bytes = a.ld_k * es;
+  p->g_mis0 = (int32_t)((uintptr_t)a.G & 15);
+  p->g_mis_m = (int32_t)((a.ld_m * es) & 15);
+  p->g_mis_k = (int32_t)((a.ld_k * es) & 15);
+}
 
 }  // namespace
 
@@ -564,25 +679,19 @@ bool encode_map(CUtensorMap *map, const void *base, int unit_bytes, int rank, co
 // apply (then the direct-load kernel runs the whole range).
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   PipeTuning &t = tuning();
-  if (!t.enabled) return false;
-  if (t.sm_count == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&t.sm_count, cudaDevAttrMultiProcessorCount, dev);
-    if (t.sm_count <= 0) t.sm_count = 148;
-  }
-  // bulk copies need 16-byte aligned sources and sizes
-  if ((uintptr_t)a.G % 16 != 0 || (a.ld_m * es) % 16 != 0 || (a.ld_k * es) % 16 != 0) return false;
+  if ((uintptr_t)a.G % es != 0) return false;
   if (!encode_fn()) return false;
   int R = t.rows ? t.rows : 8;
   if (R < 1) R = 1;
   if (R > kMaxRowsPerItem) R = kMaxRowsPerItem;
   if (R > a.M) R = a.M;
+  const bool rows_aligned = coverage(a, es, 512).rows_aligned;
+  const int row_pad = rows_aligned ? 0 : 16;
   // Tile width: a box row is 256 units of T*es/256 bytes, so T is 128, 256 or 512.
   // Shapes tried in order (measured on B200, see profiles/): two CTAs per SM with two consumer
   // groups each while the double-buffered X stage leaves room for it (K <= 16 at T = 512), else one
   // CTA per SM with four groups; then narrower tiles.  The first shape whose ring has at least two
-  // slots per group is taken.  Environment overrides replace the corresponding field of every shape.
+  // slots per group is taken.  A tuning build's overrides replace the corresponding field of every shape.
   struct Shape { int T, ctas, groups; };
   const Shape shapes[] = {{512, 2, 2}, {512, 1, 4}, {256, 1, 4}, {128, 1, 4}};
   int T = 0, ctas = 0, groups = 0, slots = 0;
@@ -596,57 +705,55 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
     if (groups > a.K) groups = a.K;
     while (groups > 1 && groups * (T / 4) > 512) --groups;
     if (groups < 1 || ctas < 1) return false;
-    const PipeLayout L0 = pipe_layout(a.K, T, es, R, 0, a.mix_slots);
+    const PipeLayout L0 = pipe_layout(a.K, T, es, R, 0, a.mix_slots, row_pad);
     const int budget = kSmemBudget / ctas - 1024;
-    slots = (budget - L0.total - 256) / (T * 4 + R * T * es);
+    slots = (budget - L0.total - 256) / slot_bytes_of(T * 4, T, es, R, row_pad);
     if (t.slots && t.slots < slots) slots = t.slots;
     if (slots > 32) slots = 32;
     slots -= slots % groups;  // every group's ring has the same number of slots
     if (slots >= 2 * groups) { found = true; break; }
   }
   if (!found) return false;
-  if ((a.P / T) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
+  const Coverage cov = coverage(a, es, T);
+  if (cov.n_tiles < 1) return false;
+  if ((cov.n_tiles + 1) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
   // When one item holds a learner's whole contribution (R >= M) two slots per group are enough to
   // keep the copies back to back, and deeper rings measured 1-4 % slower (MATCHA and all-reduce
   // workloads with M = 4); learners that need several items per tile use all the slots that fit.
   if (!t.slots && R >= a.M && slots > 2 * groups) slots = 2 * groups;
-  if (a.P < T) return false;
-  const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots);
+  const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots, row_pad);
   if (L.total > kSmemBudget) return false;
   plan->T = T;
   plan->rows_per_item = R;
   plan->n_slots = slots;
   plan->n_groups = groups;
   plan->smem_bytes = L.total;
-  plan->n_tiles = (int)(a.P / T);
+  plan->n_tiles = (int)cov.n_tiles;
+  plan->head = (int)cov.head;
+  plan->row_copies = rows_aligned ? 0 : 1;
   const int64_t max_ctas = (int64_t)ctas * t.sm_count;
   plan->grid = (int)(plan->n_tiles < max_ctas ? plan->n_tiles : max_ctas);
-  return plan->n_tiles > 0;
+  return true;
 }
 
-// Shape of the no-stage kernel: T = 512 (or narrower), R rows per item, as many CTAs per SM as
-// keep at least 3 slots per group.
+// Shape of the no-stage kernel: T = 512, R rows per item, as many CTAs per SM as keep at least
+// 2 slots per group.
 bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   PipeTuning &t = tuning();
-  if (!t.enabled) return false;
-  if (t.sm_count == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&t.sm_count, cudaDevAttrMultiProcessorCount, dev);
-    if (t.sm_count <= 0) t.sm_count = 148;
-  }
-  if ((uintptr_t)a.G % 16 != 0 || (a.ld_m * es) % 16 != 0 || (a.ld_k * es) % 16 != 0) return false;
+  if ((uintptr_t)a.G % es != 0) return false;
   if (!encode_fn()) return false;
   const int T = 512;
-  if (a.P < T) return false;
-  if ((a.P / T) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
+  const Coverage cov = coverage(a, es, T);
+  if (cov.n_tiles < 1) return false;
+  if ((cov.n_tiles + 1) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
+  const int row_pad = cov.rows_aligned ? 0 : 16;
   int R = es == 2 ? 8 : 4;
   if (R > a.M) R = a.M;
   int groups = centralized ? 1 : 2;
   if (groups > a.K) groups = a.K;
   const int ctas = centralized ? 4 : 2;
   const int budget = kSmemBudget / ctas - 1024;
-  int slots = (budget - 512) / (R * T * es);
+  int slots = (budget - 512) / slot_bytes_of(0, T, es, R, row_pad);
   if (slots > 16) slots = 16;
   slots -= slots % groups;
   if (slots < 2 * groups) return false;
@@ -654,13 +761,17 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   plan->rows_per_item = R;
   plan->n_slots = slots;
   plan->n_groups = groups;
-  plan->smem_bytes = stream_layout(T, es, R, slots).total;
-  plan->n_tiles = (int)(a.P / T);
+  plan->smem_bytes = stream_layout(T, es, R, slots, row_pad).total;
+  plan->n_tiles = (int)cov.n_tiles;
+  plan->head = (int)cov.head;
+  plan->row_copies = cov.rows_aligned ? 0 : 1;
   const int64_t max_ctas = (int64_t)ctas * t.sm_count;
   plan->grid = (int)(plan->n_tiles < max_ctas ? plan->n_tiles : max_ctas);
-  return plan->n_tiles > 0;
+  return true;
 }
 
+namespace {
+// G: [K, M, units]; one map per box height (16-byte aligned rows only).
 bool encode_gmaps(PipeArgs *p, const StepArgs &a, int es, const PipePlan &plan) {
   const cuuint64_t units = (cuuint64_t)plan.n_tiles * kBoxInner;
   const int ub = plan.T * es / kBoxInner;
@@ -674,26 +785,39 @@ bool encode_gmaps(PipeArgs *p, const StepArgs &a, int es, const PipePlan &plan) 
   return true;
 }
 
+void fill_pipe_args(PipeArgs *p, const StepArgs &a, const PipePlan &plan, int *err_flag) {
+  std::memset(p, 0, sizeof(*p));
+  p->s = a;
+  p->T = plan.T;
+  p->n_slots = plan.n_slots;
+  p->rows_per_item = plan.rows_per_item;
+  p->n_tiles = plan.n_tiles;
+  p->n_groups = plan.n_groups;
+  p->err = err_flag;
+}
+}  // namespace
+
+// `a` describes the columns the kernel covers (the caller has already cut off plan.head).
 cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, const PipePlan &plan, int *err_flag,
                                    cudaStream_t st) {
   PipeArgs p;
-  std::memset(&p, 0, sizeof(p));
-  p.s = a;
-  p.T = plan.T;
-  p.n_slots = plan.n_slots;
-  p.rows_per_item = plan.rows_per_item;
-  p.n_tiles = plan.n_tiles;
-  p.n_groups = plan.n_groups;
-  p.err = err_flag;
-  if (!encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;  // nothing launched: caller falls back
+  fill_pipe_args(&p, a, plan, err_flag);
+  if (plan.row_copies) fill_row_args(&p, a, es);
+  else if (!encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;  // nothing launched: caller falls back
   const int threads = plan.n_groups * (32 + plan.T / 4);
+#define NB_LAUNCH(ES, MODE)                                                                               \
+  do {                                                                                                    \
+    if (plan.row_copies) nb_stream_pipeline_kernel<ES, MODE, false><<<plan.grid, threads, plan.smem_bytes, st>>>(p); \
+    else nb_stream_pipeline_kernel<ES, MODE, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);       \
+  } while (0)
   if (es == 2) {
-    if (centralized) nb_stream_pipeline_kernel<2, kModeCentralized><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
-    else nb_stream_pipeline_kernel<2, kModeAccumulate><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
+    if (centralized) NB_LAUNCH(2, kModeCentralized);
+    else NB_LAUNCH(2, kModeAccumulate);
   } else {
-    if (centralized) nb_stream_pipeline_kernel<4, kModeCentralized><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
-    else nb_stream_pipeline_kernel<4, kModeAccumulate><<<plan.grid, threads, plan.smem_bytes, st>>>(p);
+    if (centralized) NB_LAUNCH(4, kModeCentralized);
+    else NB_LAUNCH(4, kModeAccumulate);
   }
+#undef NB_LAUNCH
   return cudaGetLastError();
 }
 
@@ -704,34 +828,26 @@ cudaError_t launch_wait_selftest(int *err_flag, int code, long long limit_cycles
 
 cudaError_t configure_pipeline() {
   cudaError_t e;
-#define NB_CFG(ES, MEAN)                                                                              \
-  if ((e = cudaFuncSetAttribute(nb_step_pipeline_kernel<ES, MEAN, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                kSmemBudget)) != cudaSuccess)                                         \
-    return e;                                                                                         \
-  if ((e = cudaFuncSetAttribute(nb_step_pipeline_kernel<ES, MEAN, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                kSmemBudget)) != cudaSuccess)                                         \
+#define NB_CFG1(...)                                                                                                  \
+  if ((e = cudaFuncSetAttribute(__VA_ARGS__, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget)) != cudaSuccess) \
     return e;
+#define NB_CFG(ES, MEAN)                                                                   \
+  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, true>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, true>) \
+  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, false>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, false>)
   NB_CFG(2, true) NB_CFG(2, false) NB_CFG(4, true) NB_CFG(4, false)
 #undef NB_CFG
-#define NB_CFG(ES, MODE)                                                                                          \
-  if ((e = cudaFuncSetAttribute(nb_stream_pipeline_kernel<ES, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                kSmemBudget)) != cudaSuccess)                                                     \
-    return e;
+#define NB_CFG(ES, MODE) \
+  NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, true>) NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, false>)
   NB_CFG(2, kModeAccumulate) NB_CFG(2, kModeCentralized) NB_CFG(4, kModeAccumulate) NB_CFG(4, kModeCentralized)
 #undef NB_CFG
+#undef NB_CFG1
   return cudaSuccess;
 }
 
+// `a` describes the columns the kernel covers (the caller has already cut off plan.head).
 cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan, int *err_flag, cudaStream_t st) {
   PipeArgs p;
-  std::memset(&p, 0, sizeof(p));
-  p.s = a;
-  p.T = plan.T;
-  p.n_slots = plan.n_slots;
-  p.rows_per_item = plan.rows_per_item;
-  p.n_tiles = plan.n_tiles;
-  p.n_groups = plan.n_groups;
-  p.err = err_flag;
+  fill_pipe_args(&p, a, plan, err_flag);
   const cuuint64_t units = (cuuint64_t)plan.n_tiles * kBoxInner;
   {  // X and V: [K, units] fp32 rows of pitch ldx
     const int ub = plan.T * 4 / kBoxInner;
@@ -742,12 +858,18 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
     if (!encode_map(&p.xmap, a.X, ub, 2, dims, strides, xbox) || !encode_map(&p.vmap, a.V, ub, 2, dims, strides, vbox))
       return cudaErrorNotSupported;  // nothing launched: caller falls back to the direct-load kernel
   }
-  if (!encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;  // G: [K, M, units]; one map per box height
+  if (plan.row_copies) fill_row_args(&p, a, es);
+  else if (!encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;
   const int threads = 32 + plan.n_groups * (32 + plan.T / 4);  // X producer + per group: producer warp + consumers
-#define NB_LAUNCH(ES, MEAN)                                                                                   \
-  do {                                                                                                        \
-    if (plan.T == 512) nb_step_pipeline_kernel<ES, MEAN, 512><<<plan.grid, threads, plan.smem_bytes, st>>>(p); \
-    else nb_step_pipeline_kernel<ES, MEAN, 0><<<plan.grid, threads, plan.smem_bytes, st>>>(p);                 \
+#define NB_LAUNCH2(ES, MEAN, TT)                                                                                   \
+  do {                                                                                                             \
+    if (plan.row_copies) nb_step_pipeline_kernel<ES, MEAN, TT, false><<<plan.grid, threads, plan.smem_bytes, st>>>(p); \
+    else nb_step_pipeline_kernel<ES, MEAN, TT, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);              \
+  } while (0)
+#define NB_LAUNCH(ES, MEAN)                       \
+  do {                                            \
+    if (plan.T == 512) NB_LAUNCH2(ES, MEAN, 512); \
+    else NB_LAUNCH2(ES, MEAN, 0);                 \
   } while (0)
   if (es == 2) {
     if (a.mean_mode) NB_LAUNCH(2, true);
@@ -757,6 +879,7 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
     else NB_LAUNCH(4, false);
   }
 #undef NB_LAUNCH
+#undef NB_LAUNCH2
   return cudaGetLastError();
 }
 

@@ -53,7 +53,10 @@ def _against_oracle(B, w, steps, counts=None, fused=True):
     (3 * 512, 1),
     (511, 1),            # below one tile (and unaligned): direct kernel only
     (256, 1),
-    (2 * 512 + 1, 1),    # odd row length: rows are not 16-byte aligned -> direct kernel only
+    (2 * 512 + 1, 2),    # odd row length: one tile of per-row bulk copies (the second would read past
+                         # the end of the last row) + a 513-column tail
+    (2 * 512 + 8, 2),    # rows are 16-byte multiples again: two tiles of box copies + 8 columns
+    (512 + 7, 1),        # odd and shorter than one tile plus the 16 bytes a row copy may over-read
 ])
 def test_sizes_around_one_tile(B, P, expected_launches):
     w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], P, steps=3)
@@ -115,67 +118,106 @@ def test_matcha_and_options_on_pipeline_sizes(B):
         ctx.close()
 
 
-@pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16"])
-@pytest.mark.parametrize("order", [0, 1])
-def test_pipeline_and_direct_kernels_agree_bitwise(B, name, order):
-    """The same values reach the library once as a 16-byte aligned stream (pipeline kernel + tail)
-    and once shifted by one element (rows lose their alignment, so the direct-load kernel with
-    scalar loads runs everything): identical bits."""
+def _shifted_view(g, by=1):
+    """The same values `by` elements further into a fresh buffer: rows lose their 16-byte alignment."""
     import torch
-    w = WL.scaled(WL.WORKLOADS[name], 5 * 512 + 40, steps=3)   # rows stay 16-byte multiples in bf16 too
-    a, b = B.context_for(w), B.context_for(w)
-    for c in (a, b):
+    flat = torch.empty(g.numel() + by, dtype=g.dtype, device=g.device)
+    out = flat[by:].view_as(g)
+    out.copy_(g)
+    return out
+
+
+@pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16",
+                                  "cfg5_scale_ring"])
+@pytest.mark.parametrize("order", [0, 1])
+@pytest.mark.parametrize("P", [5 * 512 + 40, 5 * 512 + 41, 5 * 512 + 44])
+def test_pipeline_and_direct_kernels_agree_bitwise(B, name, order, P):
+    """The same values reach the library four ways: as a 16-byte aligned dense stream (for P = 5*512+40
+    every row is a 16-byte multiple: box copies; for the odd P and for P = 4 mod 8 in bf16 the rows
+    are not: one bulk copy per row), shifted by one element (the stream itself starts off a 16-byte
+    boundary: the first tile goes to the direct-load kernel), shifted by three, and through the
+    direct-load kernels alone.  Identical bits every time."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS[name], P, steps=3)
+    es = 2 if w.grad_dtype == "bf16" else 4
+    rows_aligned = (P * es) % 16 == 0
+    ctxs = [B.context_for(w) for _ in range(4)]
+    a, b, b3, d = ctxs
+    d.set_option(B.NB_OPT_KERNEL, B.NB_KERNEL_DIRECT)
+    for c in ctxs:
         c.set_option(B.NB_OPT_ORDER, order)
         c.set_params(torch.from_numpy(WL.init_params(w)).cuda())
+    extra = 1 if w.variant == "matcha" else 0
     for t in range(w.steps):
         n = H.lib_counts(B, w, t)
         g = H.to_device(WL.gradients_np(w, t)[0])
-        flat = torch.empty(g.numel() + 1, dtype=g.dtype, device="cuda")
-        shifted = flat[1:].view_as(g)
-        shifted.copy_(g)
-        la = a.get_stats()["kernel_launches"]
-        a.step_fused(g, n)
-        lb = b.get_stats()["kernel_launches"]
-        b.step_fused(shifted, n)
-        extra = 1 if w.variant == "matcha" else 0
-        assert a.get_stats()["kernel_launches"] - la == 2 + extra      # pipeline + tail
-        assert b.get_stats()["kernel_launches"] - lb == 1 + extra      # direct only
-    assert torch.equal(a.get_params(), b.get_params())
-    assert torch.equal(a.get_momentum(), b.get_momentum())
-    a.close(); b.close()
+        streams = (g, _shifted_view(g, 1), _shifted_view(g, 3), g)
+        want_launches = (2, 3, 3, 1)       # pipeline + tail; head + pipeline + tail; the same; direct only
+        want_row_copies = (0 if rows_aligned else 1, 1, 1, 0)
+        for c, gs, wl, wr in zip(ctxs, streams, want_launches, want_row_copies):
+            before = c.get_stats()["kernel_launches"]
+            c.step_fused(gs, n)
+            assert c.get_stats()["kernel_launches"] - before == wl + extra
+            plan = c.get_kernel_plan()
+            assert plan["pipeline"] == (0 if c is d else 1)
+            if c is not d:
+                assert plan["row_copies"] == wr and plan["head"] == (512 if c in (b, b3) else 0)
+                assert plan["head"] + plan["tiles"] * plan["tile"] <= P
+    for c in (b, b3, d):
+        assert torch.equal(a.get_params(), c.get_params())
+        assert torch.equal(a.get_momentum(), c.get_momentum())
+    for c in ctxs:
+        c.check_guards()
+        c.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("variant", ["dpsgd", "allreduce"])
+def test_unaligned_rows_against_the_oracle(B, dtype, variant):
+    """Odd row length on the per-row bulk-copy path, several tiles per CTA's worth of columns, every
+    row at a different byte shift, checked against the oracle (not only against the other kernels)."""
+    base = WL.WORKLOADS["cfg3_dpsgd_ring_resnet50" if variant == "dpsgd" else "cfg2_allreduce_resnet18"]
+    w = replace(WL.scaled(base, 7 * 512 + 5, steps=4), grad_dtype=dtype, K=5, M=11)
+    rng = np.random.default_rng(5)
+    counts = [rng.integers(0, w.M + 1, w.K) for _ in range(w.steps)]
+    counts[0][:] = w.M
+    _against_oracle(B, w, w.steps, counts=counts)
+    _against_oracle(B, w, w.steps, counts=counts, fused=False)
 
 
 @pytest.mark.parametrize("dtype,P", [("bf16", 4 * 512 + 40), ("f32", 3 * 512 + 12), ("bf16", 512)])
 @pytest.mark.parametrize("fused", [True, False])
 def test_centralized_step_on_pipeline_sizes(B, dtype, P, fused):
-    """Alg. 3 through the no-stage pipeline kernel (aligned rows): oracle parity, and the same bits
-    as the direct-load kernel (which a one-element shift of the stream forces)."""
+    """Alg. 3 through the no-stage pipeline kernel: oracle parity, and the same bits from box copies
+    (aligned rows), per-row bulk copies (the stream shifted by one element) and the direct-load kernel."""
     import torch
     K, M = 8, 8
     rng = np.random.default_rng(11)
     x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
     a = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
     b = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
-    for c in (a, b):
+    d = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
+    d.set_option(B.NB_OPT_KERNEL, B.NB_KERNEL_DIRECT)
+    for c in (a, b, d):
         c.set_params(torch.from_numpy(x0).cuda())
     x, v = x0.astype(np.float64), np.zeros(P)
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     for t in range(4):
         G = (torch.from_numpy(rng.standard_normal((K, M, P)).astype(np.float32)) * 0.01).to(tdt).cuda()
         n = rng.integers(0, M + 1, K)
-        flat = torch.empty(G.numel() + 1, dtype=tdt, device="cuda")
-        shifted = flat[1:].view_as(G)
-        shifted.copy_(G)
+        shifted = _shifted_view(G)
         if fused:
-            a.step_fused(G, n); b.step_fused(shifted, n)
+            a.step_fused(G, n); b.step_fused(shifted, n); d.step_fused(G, n)
         else:
             a.accumulate(G, n); a.step()
             b.accumulate(shifted, n); b.step()
+            d.accumulate(G, n); d.step()
         x, v = O.step_centralized(x, v, G.float().cpu().numpy(), n.tolist(), 0.1, 0.9)
     H.assert_close(a.get_params().numpy(), x, H.TOL_SAME_INPUT)
     H.assert_close(a.get_momentum().numpy(), v, H.TOL_SAME_INPUT)
     assert torch.equal(a.get_params(), b.get_params()) and torch.equal(a.get_momentum(), b.get_momentum())
-    a.close(); b.close()
+    assert torch.equal(a.get_params(), d.get_params()) and torch.equal(a.get_momentum(), d.get_momentum())
+    a.close(); b.close(); d.close()
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
@@ -187,27 +229,32 @@ def test_accumulate_on_pipeline_sizes(B, dtype, M):
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     a = B.NbContext(K, P, M, 0.1, 0.9, "allreduce")
     b = B.NbContext(K, P, M, 0.1, 0.9, "allreduce")
+    d = B.NbContext(K, P, M, 0.1, 0.9, "allreduce")
+    d.set_option(B.NB_OPT_KERNEL, B.NB_KERNEL_DIRECT)
     G = torch.from_numpy(rng.standard_normal((K, M, P)).astype(np.float32)).to(tdt).cuda()
     n = rng.integers(0, M + 1, K)
     n[0], n[1] = 0, M
-    flat = torch.empty(G.numel() + 1, dtype=tdt, device="cuda")
-    shifted = flat[1:].view_as(G)
-    shifted.copy_(G)
+    shifted = _shifted_view(G)
     la = a.get_stats()["kernel_launches"]
     a.accumulate(G, n)
     assert a.get_stats()["kernel_launches"] - la == 2            # pipeline kernel + 24-column tail
+    lb = b.get_stats()["kernel_launches"]
     b.accumulate(shifted, n)
+    assert b.get_stats()["kernel_launches"] - lb == 3            # first tile + per-row bulk copies + tail
+    ld = d.get_stats()["kernel_launches"]
+    d.accumulate(G, n)
+    assert d.get_stats()["kernel_launches"] - ld == 1            # direct-load kernel only
     acc = a.get_accumulator()
-    assert torch.equal(acc, b.get_accumulator())
+    assert torch.equal(acc, b.get_accumulator()) and torch.equal(acc, d.get_accumulator())
     H.assert_close(acc.numpy(), O.accumulate(G.float().cpu().numpy(), n.tolist()), 2e-6)
     assert float(acc[0].abs().max()) == 0.0
-    a.close(); b.close()
+    a.close(); b.close(); d.close()
 
 
-def test_in_place_and_out_of_place_steps_interleave(B):
-    """A context may see aligned streams (in-place pipeline kernel) and unaligned ones (out-of-place
-    kernel, after which the two model arrays trade places) in any order; state and results must be
-    those of a context that only ever saw aligned streams."""
+def test_aligned_and_unaligned_streams_interleave(B):
+    """A context may see aligned streams (box copies) and unaligned ones (per-row bulk copies plus a
+    first tile on the direct-load kernel) in any order; state and results must be those of a context
+    that only ever saw aligned streams."""
     import torch
     w = WL.scaled(WL.WORKLOADS["cfg5_scale_ring"], 4 * 512 + 40, steps=6)
     ref, mix = B.context_for(w), B.context_for(w)
@@ -218,15 +265,12 @@ def test_in_place_and_out_of_place_steps_interleave(B):
         g = H.to_device(WL.gradients_np(w, t)[0])
         ref.step_fused(g, n)
         if t in (1, 2, 4):                                   # unaligned view of the same values
-            flat = torch.empty(g.numel() + 1, dtype=g.dtype, device="cuda")
-            shifted = flat[1:].view_as(g)
-            shifted.copy_(g)
-            mix.step_fused(shifted, n)
-            assert mix.get_kernel_plan()["pipeline"] == 0
+            mix.step_fused(_shifted_view(g), n)
+            assert mix.get_kernel_plan()["row_copies"] == 1 and mix.get_kernel_plan()["head"] == 512
         else:
             mix.step_fused(g, n)
-            assert mix.get_kernel_plan()["pipeline"] == 1
-        if t == 2:                                           # checkpoint right after a swap
+            assert mix.get_kernel_plan()["row_copies"] == 0 and mix.get_kernel_plan()["head"] == 0
+        if t == 2:                                           # checkpoint in between
             X, V, step = mix.get_params(), mix.get_momentum(), mix.get_step()
             mix.set_state(step, X, V)
         assert torch.equal(ref.get_params(), mix.get_params())

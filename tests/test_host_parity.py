@@ -97,7 +97,7 @@ def test_fixed_mixing_matrices_match_oracle():
         W, _ = B.mixing_matrix(topo, B.NB_DPSGD, K, 0)
         assert np.abs(W.astype(np.float64) - O.ring_W(K)).max() < 1e-7
         W, _ = B.mixing_matrix(None, B.NB_ALLREDUCE, K, 0)
-        assert np.array_equal(W.astype(np.float64), O.full_W(K))
+        assert np.abs(W.astype(np.float64) - O.full_W(K)).max() < 1e-7      # the library holds fp32(1/K)
 
 
 def test_topology_validation():

@@ -345,8 +345,9 @@ def _sync_momentum_sgd(x0, gbar_per_step, lr, mom):
 
 
 @pytest.mark.parametrize("order", ["mix_then_update", "update_then_mix"])
-def test_all_finished_full_mixing_reduces_to_synchronous_sgd(order):
-    K, M, Pdim, steps = 4, 4, 33, 10
+@pytest.mark.parametrize("K", [3, 4, 5])
+def test_all_finished_full_mixing_reduces_to_synchronous_sgd(order, K):
+    M, Pdim, steps = 4, 33, 10
     lr, mom = 0.125, 0.5          # exact in fp32
     x0 = _rand(Pdim, 1, 0.01)
     orc = O.Oracle(K, Pdim, M, lr, mom, "allreduce", order=order)
@@ -560,6 +561,42 @@ def test_probability_projection():
                for a in np.linspace(0, 1, 41) for b in np.linspace(0, 1, 41) for c in np.linspace(0, 1, 41)
                if a + b + c <= 1.2 + 1e-12)
     assert (q - target) @ (q - target) <= best + 1e-9
+
+
+def test_algebraic_connectivity_against_textbook_spectra():
+    """matcha_lambda2 is the SECOND smallest Laplacian eigenvalue of sum_j p_j L_j.  Closed forms:
+    path graph on K vertices 2 - 2 cos(pi/K) (its eigenvalues 2 - 2 cos(pi k/K) are all distinct, so
+    taking a neighbouring index fails), cycle 2 - 2 cos(2 pi/K), complete graph K; it scales
+    linearly in a common activation probability."""
+    for K in (5, 6, 9):
+        even = [[-1] * K for _ in range(2)]
+        for u in range(K - 1):                               # edges (0,1),(2,3),... and (1,2),(3,4),...
+            even[u % 2][u], even[u % 2][u + 1] = u + 1, u
+        Ls = O.matching_laplacians(even, K)
+        want = 2.0 - 2.0 * math.cos(math.pi / K)
+        assert O.matcha_lambda2(Ls, [1.0, 1.0]) == pytest.approx(want, abs=1e-12)
+        assert O.matcha_lambda2(Ls, [0.25, 0.25]) == pytest.approx(0.25 * want, abs=1e-12)
+        third = 2.0 - 2.0 * math.cos(2.0 * math.pi / K)      # the next eigenvalue of the path is different
+        assert abs(third - want) > 0.1
+    for K in (6, 8, 10):                                     # even cycle = two perfect matchings
+        cyc = [[-1] * K for _ in range(2)]
+        for u in range(K):
+            v = (u + 1) % K
+            cyc[u % 2][u], cyc[u % 2][v] = v, u
+        assert O.matcha_lambda2(O.matching_laplacians(cyc, K), [1.0, 1.0]) == \
+            pytest.approx(2.0 - 2.0 * math.cos(2.0 * math.pi / K), abs=1e-12)
+    for K in (4, 6, 8):                                      # complete graph: round-robin 1-factorisation
+        fac = []
+        for r in range(K - 1):
+            row = [-1] * K
+            row[K - 1], row[r] = r, K - 1
+            for k in range(1, K // 2):
+                u, v = (r + k) % (K - 1), (r - k) % (K - 1)
+                row[u], row[v] = v, u
+            fac.append(row)
+        Ls = O.matching_laplacians(fac, K)
+        assert np.allclose(sum(Ls), K * np.eye(K) - np.ones((K, K)))      # the union is the complete graph
+        assert O.matcha_lambda2(Ls, [1.0] * (K - 1)) == pytest.approx(float(K), abs=1e-10)
 
 
 def test_optimal_probabilities_against_grid_search():
