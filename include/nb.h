@@ -238,6 +238,14 @@ int nb_set_params(nb_ctx *c, const float *x0, int per_learner, void *stream);
 int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
                   const int32_t *finished, void *stream);
 
+/* Row pitch, in elements, at which a gradient stream of P columns of `dtype` streams fastest: the
+ * smallest multiple of 2 KB that holds P elements.  Every 512-column tile segment of every row then
+ * lies inside one 2 KB block of device memory (measured on B200, P = 138,000,000 bf16: dense rows,
+ * whose segments straddle those blocks, run 2.7 % below rows at this pitch).  Pass it as ld_m (and
+ * M * pitch, or more, as ld_k).  Purely advisory: any pitch >= P is accepted.  Returns 0 for P < 1
+ * or an unknown dtype. */
+int64_t nb_recommended_pitch(int64_t P, int dtype);
+
 /* Streaming form of step 1 (Alg. 1 inner loop as the gradients arrive): a learner hands over one
  * finished mini-batch gradient at a time.  nb_begin_iteration clears the per-learner counts and the
  * terminal signal.  nb_accumulate_minibatch adds grad[P] (device, NB_F32 or NB_BF16) to learner i's
@@ -312,13 +320,27 @@ int nb_check_guards(nb_ctx *c, void *stream);
  * about a second; when one runs out the context reports a sticky NB_ERR_CUDA.) */
 int nb_selftest_wait_timeout(nb_ctx *c, void *stream);
 
-/* Which kernel shape ran the most recent step (for reports and tests), host out plan[10]:
+/* Bounds-checked build.  A library compiled with -DNB_DEBUG (python -m paper_2211_00889_b200.build
+ * --debug writes it next to the shipped one) checks, inside every kernel, that each tile coordinate,
+ * ring slot, shared-memory offset, table index and global address it is about to use lies inside
+ * the array it belongs to; a failed check skips the access and records a code in the device error
+ * word (100 + kind), which nb_check_guards and the host-memory outputs then report as NB_ERR_CUDA.
+ * Nothing traps.  nb_debug_build returns 1 in such a library, 0 in the shipped one.  The two
+ * functions below run the kernels' own range predicates on the host (any build): 0 if the byte span
+ * [addr, addr+bytes) lies inside [lo, hi) / if 0 <= index < count, otherwise the code a kernel
+ * would have recorded. */
+int nb_debug_build(void);
+int nb_debug_span_code(uint64_t addr, uint64_t bytes, uint64_t lo, uint64_t hi);
+int nb_debug_index_code(int64_t index, int64_t count);
+
+/* Which kernel shape ran the most recent step (for reports and tests), host out plan[12]:
  * [0] 1 if the bulk-copy pipeline kernel covered the full tiles, 0 if the direct-load kernel did
  * everything; [1] tile width in columns; [2] consumer groups per CTA; [3] ring slots per CTA;
  * [4] gradient rows per ring item; [5] CTAs launched; [6] dynamic shared memory per CTA in bytes;
  * [7] tiles covered; [8] 0 if the gradient rows travelled as tensor-map boxes, 1 if as one bulk
  * copy per row (rows not 16-byte aligned); [9] columns before the first covered tile (they, and the
- * columns after [9] + [7]*[1], went to the direct-load kernel). */
+ * columns after [9] + [7]*[1], went to the direct-load kernel); [10] buffers of the old-model stage
+ * (1-3); [11] reserved, 0. */
 int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan);
 
 /* ------------------------------------------------------------------------------------------------

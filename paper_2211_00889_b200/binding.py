@@ -10,7 +10,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libnb.so")
+LIB_PATH = os.environ.get("NB_LIB_PATH") or os.path.join(_HERE, "libnb.so")
 
 NB_OK, NB_ERR_ARG, NB_ERR_STATE, NB_ERR_CUDA, NB_ERR_NOMEM, NB_ERR_UNSUPPORTED = 0, -1, -2, -3, -4, -5
 NB_ALLREDUCE, NB_DPSGD, NB_MATCHA, NB_CENTRALIZED = 0, 1, 2, 3
@@ -93,11 +93,16 @@ def _load():
         "nb_check_guards": [vp, vp],
         "nb_selftest_wait_timeout": [vp, vp],
         "nb_step_static": [i32, i64, i32, f32, f32, vp, vp, i64, vp, i32, i64, i64, P(C.c_int32), vp],
+        "nb_debug_build": [],
+        "nb_debug_span_code": [C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint64],
+        "nb_debug_index_code": [i64, i64],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
         fn.argtypes = args
         fn.restype = C.c_int
+    lib.nb_recommended_pitch.argtypes = [i64, i32]
+    lib.nb_recommended_pitch.restype = i64
     lib.nb_last_error.argtypes = [vp]
     lib.nb_last_error.restype = C.c_char_p
     return lib
@@ -109,7 +114,8 @@ EXPORTED = ["nb_straggler_sample", "nb_topology_matchings", "nb_mixing_matrix", 
             "nb_step_fused", "nb_step_fused_host", "nb_get_params", "nb_get_momentum", "nb_get_accumulator",
             "nb_get_mean_params", "nb_set_state", "nb_get_step", "nb_get_W", "nb_get_matcha_activation",
             "nb_get_device_mixing", "nb_get_stats", "nb_step_static", "nb_get_kernel_plan", "nb_check_guards", "nb_selftest_wait_timeout",
-            "nb_matcha_optimize", "nb_begin_iteration", "nb_accumulate_minibatch", "nb_get_finished", "nb_runtime_report_compute"]
+            "nb_matcha_optimize", "nb_begin_iteration", "nb_accumulate_minibatch", "nb_get_finished", "nb_runtime_report_compute",
+            "nb_debug_build", "nb_debug_span_code", "nb_debug_index_code", "nb_recommended_pitch"]
 
 
 def _i32p(a):
@@ -385,16 +391,22 @@ class NbContext:
         self._ck(lib.nb_check_guards(self._h, _stream()))
 
     def get_kernel_plan(self):
-        a = np.zeros(10, dtype=np.int32)
+        a = np.zeros(12, dtype=np.int32)
         self._ck(lib.nb_get_kernel_plan(self._h, _i32p(a)))
         keys = ("pipeline", "tile", "groups", "slots", "rows_per_item", "grid", "smem_bytes", "tiles", "row_copies",
-                "head")
+                "head", "x_buffers", "reserved")
         return dict(zip(keys, (int(v) for v in a)))
 
     def get_stats(self):
         s, b, l = C.c_int64(0), C.c_double(0), C.c_int64(0)
         self._ck(lib.nb_get_stats(self._h, C.byref(s), C.byref(b), C.byref(l)))
         return {"sum_finished": s.value, "algorithmic_bytes": b.value, "kernel_launches": l.value}
+
+
+def recommended_pitch(P, dtype):
+    """Row pitch in elements at which a [K, M, P] gradient stream of torch dtype `dtype` streams fastest."""
+    import torch
+    return int(lib.nb_recommended_pitch(P, NB_F32 if dtype == torch.float32 else NB_BF16))
 
 
 def step_static(X, V, grads, finished, P, M, lr, mom, ld_m=0, ld_k=0):

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <utility>
@@ -116,6 +117,21 @@ bool is_device_pointer(const void *p) {
   return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged;
 }
 
+// Where the context's arrays begin and end (and, when given, the caller's gradient stream): what the
+// bounds-checked build compares every address with.
+nb::bounds::Extents extents_of(const nb_ctx *c, const void *grads, int64_t ld_m, int64_t ld_k, int es) {
+  nb::bounds::Extents e;
+  e.x_lo = (uintptr_t)c->X;
+  e.x_hi = e.x_lo + c->model_bytes;
+  e.v_lo = (uintptr_t)c->V;
+  e.v_hi = e.v_lo + c->model_bytes;
+  e.acc_lo = (uintptr_t)c->acc;
+  e.acc_hi = e.acc_lo + c->acc_bytes;
+  e.g_lo = (uintptr_t)grads;
+  e.g_hi = grads ? e.g_lo + (size_t)((int64_t)(c->K - 1) * ld_k + (int64_t)(c->M - 1) * ld_m + c->P) * (size_t)es : 0;
+  return e;
+}
+
 // Validates the gradient-stream description and the finished counts; fills the step arguments.
 int fill_step_args(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k, const int32_t *finished,
                    nb::StepArgs *a, int *esize) {
@@ -146,6 +162,8 @@ int fill_step_args(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_
   a->M = c->M;
   a->g_aligned = ((uintptr_t)grads % (size_t)(4 * es) == 0) && (ld_m % 4 == 0) && (ld_k % 4 == 0);
   for (int i = 0; i < c->K; ++i) a->n[i] = finished[i];
+  a->ext = extents_of(c, grads, ld_m, ld_k, es);
+  a->err = c->d_err;
   *esize = es;
   return NB_OK;
 }
@@ -186,6 +204,7 @@ int build_device_mixing(nb_ctx *c, cudaStream_t st) {
   m.K = c->K;
   m.n_matchings = c->mx.n_matchings;
   m.alpha = c->mx.alpha;
+  m.err = c->d_err;
   NB_CUDA(c, nb::launch_matcha_build(m, st));
   c->launches++;
   c->device_mix_valid = true;
@@ -273,6 +292,9 @@ int nb_create(nb_ctx **out, int K, int64_t P, int M, float lr, float mom, int va
   // Row pitch of X, V and acc: a multiple of the 512-column tile (2 KB), so that every row segment a
   // tile copies starts on a 2 KB boundary (measured: 2-3 % more bandwidth than 128-byte multiples).
   c->ldx = (P + 511) / 512 * 512;
+#ifdef NB_TUNING
+  if (const char *pad = std::getenv("NB_LDX_PAD")) c->ldx += 512 * (int64_t)std::atoi(pad);  // sweeps of the row pitch
+#endif
   c->mx = mx;
 
   auto bail = [&](cudaError_t e, const char *what) {
@@ -426,8 +448,10 @@ int nb_accumulate_minibatch(nb_ctx *c, int learner, const void *grad, int dtype,
   if (c->terminal) return NB_ABANDONED;  // the first finisher has ended the iteration
   const int es = dtype == NB_F32 ? 4 : 2;
   const bool aligned = (uintptr_t)grad % (size_t)(4 * es) == 0;
+  if ((uintptr_t)grad % (size_t)es != 0) return fail(c, NB_ERR_ARG, "grad is not aligned to its element size");
   NB_CUDA(c, nb::launch_add_minibatch(c->acc + (int64_t)learner * c->ldx, grad, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16,
-                                      aligned, c->P, c->n_acc[learner] == 0, (cudaStream_t)stream));
+                                      aligned, c->P, c->n_acc[learner] == 0, extents_of(c, nullptr, 0, 0, es), c->d_err,
+                                      (cudaStream_t)stream));
   c->launches++;
   c->acc_esize = es;
   if (++c->n_acc[learner] == c->M) c->terminal = true;
@@ -461,6 +485,8 @@ int nb_step(nb_ctx *c, void *stream) {
   a.K = c->K;
   a.M = c->M;
   a.g_aligned = 1;
+  a.ext = extents_of(c, nullptr, 0, 0, 4);
+  a.err = c->d_err;
   std::memcpy(a.n, c->n_acc, sizeof(a.n));
   record_stats(c, a, c->acc_esize);
   return run_update(c, &a, nb::kSrcAcc, (cudaStream_t)stream);
@@ -555,7 +581,7 @@ int nb_step_fused_host(nb_ctx *c, const void *grads_host, int dtype, int64_t ld_
     rc = launch_update(c, nb::column_range(a, c0, cols, esz), src_kind, st);
     if (rc != NB_OK) return rc;
     if (mean_out) {
-      NB_CUDA(c, nb::launch_mean(c->X + c0, c->ldx, c->rows, cols, c->d_mean + c0, st));
+      NB_CUDA(c, nb::launch_mean(c->X + c0, c->ldx, c->rows, cols, c->d_mean + c0, a.ext, c->d_err, st));
       c->launches++;
       NB_CUDA(c, cudaEventRecord(c->ev_done[q], st));
       NB_CUDA(c, cudaStreamWaitEvent(c->s_out, c->ev_done[q], 0));
@@ -593,7 +619,7 @@ int nb_get_mean_params(nb_ctx *c, float *dst, void *stream) {
     if (!c->d_mean) NB_CUDA(c, cudaMalloc(&c->d_mean, sizeof(float) * (size_t)c->P));
     out = c->d_mean;
   }
-  NB_CUDA(c, nb::launch_mean(c->X, c->ldx, c->rows, c->P, out, st));
+  NB_CUDA(c, nb::launch_mean(c->X, c->ldx, c->rows, c->P, out, extents_of(c, nullptr, 0, 0, 4), c->d_err, st));
   c->launches++;
   if (!dev) {
     NB_CUDA(c, cudaMemcpyAsync(dst, out, sizeof(float) * (size_t)c->P, cudaMemcpyDeviceToHost, st));
@@ -700,6 +726,28 @@ int nb_selftest_wait_timeout(nb_ctx *c, void *stream) {
   return NB_OK;
 }
 
+int64_t nb_recommended_pitch(int64_t P, int dtype) {
+  if (P < 1 || (dtype != NB_F32 && dtype != NB_BF16)) return 0;
+  const int64_t per_block = 2048 / (dtype == NB_F32 ? 4 : 2);
+  return (P + per_block - 1) / per_block * per_block;
+}
+
+int nb_debug_build(void) {
+#ifdef NB_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+int nb_debug_span_code(uint64_t addr, uint64_t bytes, uint64_t lo, uint64_t hi) {
+  return nb::bounds::span_code((uintptr_t)addr, bytes, (uintptr_t)lo, (uintptr_t)hi, nb::bounds::kStateAddress);
+}
+
+int nb_debug_index_code(int64_t index, int64_t count) {
+  return nb::bounds::index_inside(index, count) ? nb::bounds::kOk : nb::bounds::kLearnerIndex;
+}
+
 int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan) {
   if (!c || !plan) return NB_ERR_ARG;
   const nb::PipePlan &p = c->last_plan;
@@ -713,6 +761,8 @@ int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan) {
   plan[7] = p.n_tiles;
   plan[8] = p.row_copies;
   plan[9] = p.head;
+  plan[10] = p.x_stages;
+  plan[11] = 0;
   return NB_OK;
 }
 

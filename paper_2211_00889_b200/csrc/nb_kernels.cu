@@ -44,11 +44,7 @@ __device__ __forceinline__ float4 gather(const StepArgs &a, int i, int64_t col0,
 #pragma unroll
       for (int u = 0; u < kChunk; ++u)
         if (m0 + u < n) {
-          const float4 g = widen(r[u]);
-          acc.x = __fadd_rn(acc.x, g.x);
-          acc.y = __fadd_rn(acc.y, g.y);
-          acc.z = __fadd_rn(acc.z, g.z);
-          acc.w = __fadd_rn(acc.w, g.w);
+          acc = add4(acc, widen(r[u]));
         }
     }
     return acc;
@@ -64,6 +60,10 @@ __global__ void __launch_bounds__(256) nb_accumulate_kernel(const __grid_constan
   if (col0 >= a.P) return;
   const int nvalid = (a.P - col0 < 4) ? (int)(a.P - col0) : 4;
   const int i = blockIdx.y;
+  if constexpr (kDebug) {
+    if (!dbg_check(bounds::index_inside(i, a.K), a.err, bounds::kLearnerIndex)) return;
+    if (!dbg_thread_footprint(a, col0, nvalid, 0, i, 1, true, SRC == kSrcBF16 ? 2 : 4)) return;
+  }
   const float4 g = gather<SRC, ALIGNED>(a, i, col0, nvalid);
   st4(a.acc + (int64_t)i * a.ldx + col0, g);
 }
@@ -71,11 +71,15 @@ __global__ void __launch_bounds__(256) nb_accumulate_kernel(const __grid_constan
 // Streaming accumulate: acc_row = (first ? +0 : acc_row) + g, one mini-batch gradient at a time
 // (the same sum, in the same order, as nb_accumulate_kernel builds in one go).
 template <int SRC, bool ALIGNED>
-__global__ void __launch_bounds__(256) nb_add_minibatch_kernel(float *acc_row, const void *g, int64_t P, int first) {
+__global__ void __launch_bounds__(256) nb_add_minibatch_kernel(float *acc_row, const void *g, int64_t P, int first,
+                                                               uintptr_t acc_lo, uintptr_t acc_hi, int *err) {
   const int64_t col0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * kColsPerThread;
   if (col0 >= P) return;
   const int nvalid = (P - col0 < 4) ? (int)(P - col0) : 4;
   using E = typename ElemOf<SRC>::type;
+  if constexpr (kDebug) {  // the gradient vector is the caller's: only its length P is known, and col0 < P holds
+    if (!dbg_check(dbg_rows_inside(acc_row, 0, 1, col0, 4, 4, acc_lo, acc_hi), err, bounds::kStateAddress)) return;
+  }
   const float4 r = widen(load_raw<ALIGNED>(reinterpret_cast<const E *>(g) + col0, nvalid, (Raw<SRC> *)nullptr));
   float4 a = first ? make_float4(0.f, 0.f, 0.f, 0.f) : ld4(acc_row + col0);
   st4(acc_row + col0, add4(a, r));
@@ -115,6 +119,16 @@ __global__ void __launch_bounds__(256) nb_step_kernel(const __grid_constant__ St
   const int64_t col0 = ((int64_t)blockIdx.x * tpb + tid) * kColsPerThread;
   if (col0 >= a.P) return;
   const int nvalid = (a.P - col0 < 4) ? (int)(a.P - col0) : 4;
+  if constexpr (kDebug) {
+    if (!dbg_thread_footprint(a, col0, nvalid, K, 0, SRC == kSrcAcc ? K : 0, SRC != kSrcAcc, SRC == kSrcBF16 ? 2 : 4))
+      return;
+    if constexpr (!MEAN) {  // every column index of the staged table names a learner
+      bool tab_ok = true;
+      for (int i = 0; i < K; ++i) tab_ok = tab_ok && s_beg[i] >= 0 && s_beg[i] <= s_end[i] && s_end[i] <= a.mix_slots;
+      for (int e = 0; e < a.mix_slots; ++e) tab_ok = tab_ok && bounds::index_inside(s_col[e], K);
+      if (!dbg_check(tab_ok, a.err, bounds::kLearnerIndex)) return;
+    }
+  }
   float *Xc = a.X + col0;
   float *Vc = a.V + col0;
   const int64_t ldx = a.ldx;
@@ -169,14 +183,15 @@ __global__ void __launch_bounds__(256) nb_centralized_kernel(const __grid_consta
   const int64_t col0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * kColsPerThread;
   if (col0 >= a.P) return;
   const int nvalid = (a.P - col0 < 4) ? (int)(a.P - col0) : 4;
+  if constexpr (kDebug) {
+    if (!dbg_thread_footprint(a, col0, nvalid, 1, 0, SRC == kSrcAcc ? a.K : 0, SRC != kSrcAcc, SRC == kSrcBF16 ? 2 : 4))
+      return;
+  }
   float4 gs = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int i = 0; i < a.K; ++i) {
     const float4 g = gather<SRC, ALIGNED>(a, i, col0, nvalid);
     const float s = a.s[i];
-    gs.x = __fmaf_rn(s, g.x, gs.x);
-    gs.y = __fmaf_rn(s, g.y, gs.y);
-    gs.z = __fmaf_rn(s, g.z, gs.z);
-    gs.w = __fmaf_rn(s, g.w, gs.w);
+    gs = fma4(s, g, gs);
   }
   const float4 v = ld4(a.V + col0);
   const float4 x = ld4(a.X + col0);
@@ -200,6 +215,13 @@ __global__ void nb_matcha_build_kernel(const __grid_constant__ MatchaArgs a) {
       const int v = a.partner[c * a.K + i];
       if (((bits >> c) & 1u) && v >= 0) {
         ++cnt;
+        if constexpr (kDebug) {
+          if (!dbg_check(bounds::index_inside(e + cnt, NB_MAX_NNZ) && bounds::index_inside(v, a.K), a.err,
+                         bounds::kLearnerIndex)) {
+            --cnt;
+            continue;
+          }
+        }
         a.mix->col[e + cnt] = v;
         a.mix->val[e + cnt] = a.alpha;
       }
@@ -216,9 +238,13 @@ __global__ void nb_matcha_build_kernel(const __grid_constant__ MatchaArgs a) {
 }
 
 // Average of the learners' models (Alg. 1 / Alg. 2 "Output"), ascending learner order.
-__global__ void __launch_bounds__(256) nb_mean_kernel(const float *X, int64_t ldx, int K, int64_t P, float *out) {
+__global__ void __launch_bounds__(256) nb_mean_kernel(const float *X, int64_t ldx, int K, int64_t P, float *out,
+                                                      uintptr_t x_lo, uintptr_t x_hi, int *err) {
   const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (p >= P) return;
+  if constexpr (kDebug) {
+    if (!dbg_check(dbg_rows_inside(X, ldx, K, p, 1, 4, x_lo, x_hi), err, bounds::kStateAddress)) return;
+  }
   float s = 0.f;
   for (int i = 0; i < K; ++i) s = __fadd_rn(s, X[(int64_t)i * ldx + p]);
   out[p] = __fdiv_rn(s, (float)K);
@@ -274,6 +300,8 @@ StepArgs acc_as_stream(const StepArgs &a) {
   p.ld_k = a.ldx;
   p.M = 1;
   for (int i = 0; i < a.K; ++i) p.n[i] = 1;
+  p.ext.g_lo = a.ext.acc_lo;
+  p.ext.g_hi = a.ext.acc_hi;
   return p;
 }
 }  // namespace
@@ -402,15 +430,18 @@ cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *e
 }
 
 cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,
-                                 cudaStream_t st) {
+                                 const bounds::Extents &ext, int *err, cudaStream_t st) {
   const unsigned grid = (unsigned)((P + 1023) / 1024);
+#define NB_ADD(SRC, AL) \
+  nb_add_minibatch_kernel<SRC, AL><<<grid, 256, 0, st>>>(acc_row, g, P, first, ext.acc_lo, ext.acc_hi, err)
   if (src == kSrcF32) {
-    if (aligned) nb_add_minibatch_kernel<kSrcF32, true><<<grid, 256, 0, st>>>(acc_row, g, P, first);
-    else nb_add_minibatch_kernel<kSrcF32, false><<<grid, 256, 0, st>>>(acc_row, g, P, first);
+    if (aligned) NB_ADD(kSrcF32, true);
+    else NB_ADD(kSrcF32, false);
   } else {
-    if (aligned) nb_add_minibatch_kernel<kSrcBF16, true><<<grid, 256, 0, st>>>(acc_row, g, P, first);
-    else nb_add_minibatch_kernel<kSrcBF16, false><<<grid, 256, 0, st>>>(acc_row, g, P, first);
+    if (aligned) NB_ADD(kSrcBF16, true);
+    else NB_ADD(kSrcBF16, false);
   }
+#undef NB_ADD
   return cudaGetLastError();
 }
 
@@ -419,9 +450,10 @@ cudaError_t launch_matcha_build(const MatchaArgs &a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, cudaStream_t st) {
+cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, const bounds::Extents &ext, int *err,
+                        cudaStream_t st) {
   const unsigned grid = (unsigned)((P + 255) / 256);
-  nb_mean_kernel<<<grid, 256, 0, st>>>(X, ldx, K, P, out);
+  nb_mean_kernel<<<grid, 256, 0, st>>>(X, ldx, K, P, out, ext.x_lo, ext.x_hi, err);
   return cudaGetLastError();
 }
 

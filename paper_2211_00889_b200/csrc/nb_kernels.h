@@ -5,6 +5,7 @@
 #include <cstdint>
 
 #include "nb.h"
+#include "nb_bounds.h"
 
 namespace nb {
 
@@ -38,6 +39,9 @@ struct StepArgs {
   float lr, mom, inv_K;
   int32_t n[NB_MAX_K]; // finished counts
   float s[NB_MAX_K];   // per-learner scale (1/n_i or n_i/M)
+  // bounds-checked build only: where the arrays begin and end, and the word a failed check reports to
+  bounds::Extents ext;
+  int *err;
 };
 
 struct MatchaArgs {
@@ -48,6 +52,7 @@ struct MatchaArgs {
   int64_t step;
   int32_t K, n_matchings;
   float alpha;
+  int *err;  // bounds-checked build only: where a failed check reports to
 };
 
 // Bulk-copy pipeline kernel (nb_pipeline.cu)
@@ -55,6 +60,7 @@ struct PipePlan {
   int T, rows_per_item, n_slots, n_groups, smem_bytes, n_tiles, grid;  // all 0: the pipeline kernel did not run
   int head;        // columns [0, head) left to the direct-load kernel (a stream whose start is not 16-byte aligned)
   int row_copies;  // 0: gradient rows travel as tensor-map boxes; 1: one bulk copy per row (rows not 16-byte aligned)
+  int x_stages;    // buffers of the step kernel's X stage (0 for the kernels that have none)
 };
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan);
 bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan);
@@ -79,10 +85,11 @@ cudaError_t launch_step(const StepArgs &a, int src, bool pipeline, int *err_flag
 // The direct-load step kernel on all P columns (no pipeline kernel, no device error word).
 cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st);
 cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,
-                                 cudaStream_t st);
+                                 const bounds::Extents &ext, int *err, cudaStream_t st);
 cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, cudaStream_t st);
 cudaError_t launch_matcha_build(const MatchaArgs &a, cudaStream_t st);
-cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, cudaStream_t st);
+cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, const bounds::Extents &ext, int *err,
+                        cudaStream_t st);
 cudaError_t configure_kernels();
 
 }  // namespace nb

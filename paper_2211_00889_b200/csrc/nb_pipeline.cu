@@ -130,6 +130,7 @@ __device__ __forceinline__ void drain_and_exit_delay() {
   }
 }
 
+constexpr int kSmemBudget = 227 * 1024;
 constexpr int kMaxRowsPerItem = 8;
 constexpr int kMaxGroups = 4;
 constexpr int kBoxInner = 256;  // a box is at most 256 elements wide: rows are described in units of T*es/256 bytes
@@ -141,6 +142,7 @@ struct PipeArgs {
   int32_t rows_per_item;  // gradient rows per ring item (R)
   int32_t n_tiles;        // full tiles covered by the kernel
   int32_t n_groups;       // consumer groups (each T/4 threads)
+  int32_t x_stages;       // buffers of the X stage: 1, 2 or 3
   int *err;               // device word: 0, or the code of the wait that ran out
   // GA = false only: the gradient stream as bytes; (address & 15) of G and of the two pitches
   const unsigned char *g_base;
@@ -201,6 +203,28 @@ __device__ __forceinline__ float4 sum_rows(float4 acc, const unsigned char *rowp
   }
 }
 
+// Bounds-checked build: everything the producer is about to use for one ring item - the slot, the
+// copy coordinates, and (per-row copies) the source span of this lane's row - is in range.
+template <int ES, bool GA>
+__device__ __forceinline__ bool dbg_item_ok(const PipeArgs &a, int T, int tile, int i, int m0, int rows, int lane,
+                                            uint32_t sl, int NS, int off_slots, int slot_bytes, int total) {
+  bool ok = dbg_check(sl < (uint32_t)NS && off_slots + (int)(sl + 1) * slot_bytes <= total, a.err, bounds::kRingSlot);
+  ok = dbg_check(bounds::index_inside(tile, a.n_tiles) && bounds::index_inside(i, a.s.K) && m0 >= 0 && rows >= 0 &&
+                     m0 + rows <= a.s.M && rows <= kMaxRowsPerItem,
+                 a.err, bounds::kTileCoordinate) && ok;
+  if constexpr (!GA) {
+    if (lane < rows) {
+      const unsigned char *src = a.g_base + (int64_t)i * a.g_ld_k_bytes + (int64_t)(m0 + lane) * a.g_ld_m_bytes +
+                                 (int64_t)tile * (T * ES);
+      src -= reinterpret_cast<uintptr_t>(src) & 15;
+      ok = dbg_check(bounds::span_inside(reinterpret_cast<uintptr_t>(src), (uint64_t)(T * ES + 16), a.s.ext.g_lo,
+                                         a.s.ext.g_hi),
+                     a.err, bounds::kGradientAddress) && ok;
+    }
+  }
+  return ok;
+}
+
 // Producer side of one ring item's gradient rows.  GA: lane 0 issues one box of exactly `rows` rows.
 // Otherwise lanes 0..rows-1 each fetch the aligned superset of one row's tile segment.
 template <int ES, bool GA>
@@ -229,15 +253,17 @@ struct PipeLayout {
 };
 
 // row_pad: 0 for box copies, 16 when every row is staged as its 16-byte aligned superset.
-__host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, int n_slots, int mix_slots, int row_pad) {
+constexpr int kMaxXStages = 3;
+__host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, int n_slots, int mix_slots, int row_pad,
+                                                  int x_stages) {
   PipeLayout L;
-  int off = (2 * n_slots + 5) * 8;
+  int off = (2 * n_slots + 3 * kMaxXStages) * 8;
   off = (off + 127) / 128 * 128;
   L.off_tab = off;
   off += mix_slots * 8 + K * 8;
   off = (off + 127) / 128 * 128;
   L.off_xs = off;
-  off += 2 * K * T * 4;  // the X stage is double-buffered: tile t+1's models load while tile t is consumed
+  off += x_stages * K * T * 4;  // two buffers: tile t+1's models load while tile t is consumed (see the kernel)
   L.off_slots = off;
   L.slot_bytes = slot_bytes_of(T * 4, T, es, R, row_pad);
   L.total = off + n_slots * L.slot_bytes;
@@ -255,17 +281,18 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
   const StepArgs &s = a.s;
   const int K = s.K, T = TT ? TT : a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
   const int NSG = NS / NG;  // slots in each group's ring
-  const PipeLayout L = pipe_layout(K, T, ES, R, NS, s.mix_slots, kRowPad);
+  const int NXS = a.x_stages;
+  const PipeLayout L = pipe_layout(K, T, ES, R, NS, s.mix_slots, kRowPad, NXS);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);
   uint64_t *empty = full + NS;
   uint64_t *xfull = empty + NS;
-  uint64_t *xempty = xfull + 2;
-  uint64_t *ybar = xfull + 4;
+  uint64_t *xempty = xfull + kMaxXStages;
+  uint64_t *ybar = xempty + kMaxXStages;
   int32_t *s_col = reinterpret_cast<int32_t *>(smem_raw + L.off_tab);
   float *s_val = reinterpret_cast<float *>(s_col + s.mix_slots);
   int32_t *s_beg = reinterpret_cast<int32_t *>(s_val + s.mix_slots);
   int32_t *s_end = s_beg + K;
-  float *xs_base = reinterpret_cast<float *>(smem_raw + L.off_xs);  // two stages of K*T floats
+  float *xs_base = reinterpret_cast<float *>(smem_raw + L.off_xs);  // NXS buffers of K*T floats
   unsigned char *slots = smem_raw + L.off_slots;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -276,24 +303,31 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
       mbar_init(&full[q], 1);
       mbar_init(&empty[q], group_warps);            // released by the group that owns the ring
     }
-    for (int q = 0; q < 2; ++q) {
+    for (int q = 0; q < kMaxXStages; ++q) {
       mbar_init(&xfull[q], 1);
       mbar_init(&xempty[q], n_cons_warps);
+      mbar_init(&ybar[q], n_cons_warps);
     }
-    mbar_init(ybar, n_cons_warps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  bool table_ok = true;
   if constexpr (!MEAN) {
     for (int e = threadIdx.x; e < s.mix_slots; e += blockDim.x) {
       s_col[e] = s.mix->col[e];
       s_val[e] = s.mix->val[e];
+      if constexpr (kDebug) table_ok = table_ok && bounds::index_inside(s_col[e], K);
     }
     for (int e = threadIdx.x; e < K; e += blockDim.x) {
       s_beg[e] = s.mix->row_beg[e];
       s_end[e] = s.mix->row_end[e];
+      if constexpr (kDebug) table_ok = table_ok && s_beg[e] >= 0 && s_beg[e] <= s_end[e] && s_end[e] <= s.mix_slots;
     }
   }
-  __syncthreads();
+  if constexpr (kDebug) {  // a table entry that names no learner: the whole CTA leaves before touching anything
+    if (__syncthreads_or(!dbg_check(table_ok && L.total <= kSmemBudget, a.err, bounds::kLearnerIndex))) return;
+  } else {
+    __syncthreads();
+  }
 
   const int64_t ldx = s.ldx;
   bool ok = true;
@@ -317,6 +351,11 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
             if constexpr (GA) ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2);
             else ok = __all_sync(0xffffffffu, mbar_wait(&empty[sl], phase ^ 1, a.err, 2));
             if (!ok) break;
+            if constexpr (kDebug) {
+              ok = dbg_item_ok<ES, GA>(a, T, tile, i, m0, rows, lane, sl, NS, L.off_slots, L.slot_bytes, L.total);
+              if constexpr (!GA) ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+            }
             unsigned char *dst = slots + (size_t)sl * L.slot_bytes;
             if (lane == 0) {
               mbar_expect_tx(&full[sl], (uint32_t)(rows * (T * ES + kRowPad) + (m0 == 0 ? T * 4 : 0)));
@@ -331,16 +370,24 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
       }
     }
   } else if (warp == NG) {
-    // ------------------------------------------- X producer: the tiles' old models, two stages
-    // Stage b = titer & 1 is reused every second tile; its k-th use waits for the (k-1)-th release,
-    // so tile t+1's models load while tile t is consumed.
+    // ------------------------------------------- X producer: the tiles' old models, NXS buffers
+    // Buffer b = titer % NXS is reused every NXS-th tile; its k-th use waits for the (k-1)-th
+    // release, so with two buffers tile t+1's models load while tile t is consumed.  (One buffer:
+    // K so large that two do not fit; the ring keeps filling while the next tile's models load.
+    // Three: the update-then-mix order, whose averaging pass runs one tile late.)
     if (lane == 0) {
-      int titer = 0;
+      int titer = 0, b = 0;
+      uint32_t xpar = 0;
       for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x, ++titer) {
-        const int b = titer & 1;
-        if (!(ok = mbar_wait(&xempty[b], ((titer >> 1) & 1) ^ 1, a.err, 1))) break;
+        if (!(ok = mbar_wait(&xempty[b], xpar ^ 1, a.err, 1))) break;
+        if constexpr (kDebug) {
+          if (!(ok = dbg_check(bounds::index_inside(tile, a.n_tiles) && L.off_xs + (b + 1) * K * T * 4 <= L.off_slots,
+                               a.err, bounds::kTileCoordinate)))
+            break;
+        }
         mbar_expect_tx(&xfull[b], (uint32_t)(K * T * 4));
         tma_load_2d(xs_base + (size_t)b * K * T, &a.xmap, tile * kBoxInner, 0, &xfull[b]);
+        if (++b == NXS) { b = 0; xpar ^= 1; }
       }
     }
   } else {
@@ -353,17 +400,55 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
     {
       const float lr = s.lr, mom = s.mom;
       const bool mix_first = s.order == NB_ORDER_MIX_THEN_UPDATE;
+      // Update-then-mix (Eq. 4-6) needs every learner's y_j = x_j - lr v_j of the tile before anyone
+      // averages, so the tile has two passes with a rendezvous of all groups in between.  With three
+      // X buffers the averaging pass of tile t runs after the first pass of tile t+1: the groups
+      // reach the rendezvous with a tile of slack and nobody idles at it.
+      const bool defer = !mix_first && NXS >= 3;
+
+      // Second pass of update-then-mix on buffer ub (columns at ucol0): x_i = sum_j W_ij y_j.
+      auto average_and_store = [&](int ub, uint32_t upar, int64_t ucol0) -> bool {
+        if (!__all_sync(0xffffffffu, mbar_wait(&ybar[ub], upar, a.err, 5))) return false;
+        const float4 *ys4 = reinterpret_cast<const float4 *>(xs_base + (size_t)ub * K * T);
+        float *Xu = s.X + ucol0;
+        float4 mean = make_float4(0.f, 0.f, 0.f, 0.f);
+        if constexpr (MEAN) {
+          for (int j = 0; j < K; ++j) mean = add4(mean, ys4[j * nq + cq]);
+          mean = scale4(mean, s.inv_K);
+        }
+        for (int i = grp; i < K; i += NG) {
+          float4 xn;
+          if constexpr (MEAN) xn = mean;
+          else xn = mix_row(ys4, nq, cq, s_col, s_val, s_beg[i], s_end[i]);
+          st4(Xu + (int64_t)i * ldx, xn);
+        }
+        // the buffer was written through the generic proxy; order that before the next bulk copy
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&xempty[ub]);
+        return true;
+      };
+
       uint32_t slot = 0, phase = 0;
-      int titer = 0;
+      int titer = 0, xb = 0, prev_xb = 0;
+      uint32_t xpar = 0, prev_xpar = 0;
+      int64_t prev_col0 = 0;
       for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x, ++titer) {
         const int64_t col0 = (int64_t)tile * T + (int64_t)cq * 4;
         float *Xc = s.X + col0;
         float *Vc = s.V + col0;
-        const int xb = titer & 1;
         float4 *xs4w = reinterpret_cast<float4 *>(xs_base + (size_t)xb * K * T);
         const float4 *xs4 = xs4w;
-        ok = __all_sync(0xffffffffu, mbar_wait(&xfull[xb], (titer >> 1) & 1, a.err, 3));  // warp-uniform outcome
+        ok = __all_sync(0xffffffffu, mbar_wait(&xfull[xb], xpar, a.err, 3));  // warp-uniform outcome
         if (!ok) break;
+        if constexpr (kDebug) {  // this thread's stores of the tile: 4 columns of all K rows of X and V
+          ok = __all_sync(0xffffffffu,
+                          dbg_check(dbg_rows_inside(s.X, ldx, K, col0, 4, 4, s.ext.x_lo, s.ext.x_hi) &&
+                                        dbg_rows_inside(s.V, ldx, K, col0, 4, 4, s.ext.v_lo, s.ext.v_hi) &&
+                                        bounds::index_inside(xb, NXS),
+                                    a.err, bounds::kStateAddress));
+          if (!ok) break;
+        }
         float4 mean = make_float4(0.f, 0.f, 0.f, 0.f);
         if (MEAN && mix_first) {
           for (int j = 0; j < K; ++j) mean = add4(mean, xs4[j * nq + cq]);
@@ -379,6 +464,11 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
             const uint32_t sl = (uint32_t)grp * NSG + slot;
             ok = __all_sync(0xffffffffu, mbar_wait(&full[sl], phase, a.err, 4));
             if (!ok) break;
+            if constexpr (kDebug) {
+              ok = __all_sync(0xffffffffu, dbg_check(sl < (uint32_t)NS && L.off_slots + (int)(sl + 1) * L.slot_bytes <= L.total,
+                                                     a.err, bounds::kRingSlot));
+              if (!ok) break;
+            }
             const unsigned char *src = slots + (size_t)sl * L.slot_bytes;
             if (m0 == 0) v = reinterpret_cast<const float4 *>(src)[cq];
             const int s0 = GA ? 0 : (a.g_mis0 + i * a.g_mis_k + m0 * a.g_mis_m);
@@ -397,32 +487,29 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
             else xh = mix_row(xs4, nq, cq, s_col, s_val, s_beg[i], s_end[i]);
             st4(Xc + (int64_t)i * ldx, descend(xh, lr, vn));
           } else {
-            xs4w[i * nq + cq] = descend(xs4[i * nq + cq], lr, vn);  // y_i replaces x_i in the stage
+            xs4w[i * nq + cq] = descend(xs4[i * nq + cq], lr, vn);  // y_i replaces x_i in the buffer
           }
         }
         if (!ok) break;
-        if (!mix_first) {
-          // every group's y must be staged before anyone averages: bounded mbarrier rendezvous
+        if (mix_first) {
           __syncwarp();
-          if (lane == 0) mbar_arrive(ybar);
-          ok = __all_sync(0xffffffffu, mbar_wait(ybar, titer & 1, a.err, 5));
-          if (!ok) break;
-          if constexpr (MEAN) {
-            for (int j = 0; j < K; ++j) mean = add4(mean, xs4[j * nq + cq]);
-            mean = scale4(mean, s.inv_K);
+          if (lane == 0) mbar_arrive(&xempty[xb]);
+        } else {
+          // this group's y of the tile are staged: tell the others (bounded mbarrier rendezvous)
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&ybar[xb]);
+          if (!defer) {
+            if (!(ok = average_and_store(xb, xpar, col0))) break;
+          } else if (titer > 0) {
+            if (!(ok = average_and_store(prev_xb, prev_xpar, prev_col0))) break;
           }
-          for (int i = grp; i < K; i += NG) {
-            float4 xn;
-            if constexpr (MEAN) xn = mean;
-            else xn = mix_row(xs4, nq, cq, s_col, s_val, s_beg[i], s_end[i]);
-            st4(Xc + (int64_t)i * ldx, xn);
-          }
-          // the stage was written through the generic proxy; order that before the next bulk copy
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          prev_xb = xb;
+          prev_xpar = xpar;
+          prev_col0 = col0;
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&xempty[xb]);
+        if (++xb == NXS) { xb = 0; xpar ^= 1; }
       }
+      if (ok && defer && titer > 0) ok = average_and_store(prev_xb, prev_xpar, prev_col0);  // the last tile's second pass
     }
   }
   if (!ok) drain_and_exit_delay();
@@ -490,6 +577,11 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
             if constexpr (GA) ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2);
             else ok = __all_sync(0xffffffffu, mbar_wait(&empty[sl], phase ^ 1, a.err, 2));
             if (!ok) break;
+            if constexpr (kDebug) {
+              ok = dbg_item_ok<ES, GA>(a, T, tile, i, m0, rows, lane, sl, NS, L.off_slots, L.slot_bytes, L.total);
+              if constexpr (!GA) ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+            }
             if (lane == 0) mbar_expect_tx(&full[sl], (uint32_t)(rows * (T * ES + kRowPad)));  // 0 rows: a plain arrival
             if constexpr (!GA) __syncwarp();
             issue_rows<ES, GA>(a, slots + (size_t)sl * L.slot_bytes, T, tile, i, m0, rows, lane, &full[sl]);
@@ -507,6 +599,14 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
     for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x) {
       const int64_t col0 = (int64_t)tile * T + (int64_t)cq * 4;
       float4 x = make_float4(0.f, 0.f, 0.f, 0.f), v = x, gs = x;
+      if constexpr (kDebug) {  // this thread's global footprint of the tile
+        const bool in = MODE == kModeAccumulate
+                            ? dbg_rows_inside(s.acc, ldx, K, col0, 4, 4, s.ext.acc_lo, s.ext.acc_hi)
+                            : dbg_rows_inside(s.X, ldx, 1, col0, 4, 4, s.ext.x_lo, s.ext.x_hi) &&
+                                  dbg_rows_inside(s.V, ldx, 1, col0, 4, 4, s.ext.v_lo, s.ext.v_hi);
+        ok = __all_sync(0xffffffffu, dbg_check(in, a.err, bounds::kStateAddress));
+        if (!ok) break;
+      }
       if constexpr (MODE == kModeCentralized) {  // requested early, used after the last learner
         x = ld4(s.X + col0);
         v = ld4(s.V + col0);
@@ -520,6 +620,11 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
           const uint32_t sl = (uint32_t)grp * NSG + slot;
           ok = __all_sync(0xffffffffu, mbar_wait(&full[sl], phase, a.err, 4));
           if (!ok) break;
+          if constexpr (kDebug) {
+            ok = __all_sync(0xffffffffu, dbg_check(sl < (uint32_t)NS && L.off_slots + (int)(sl + 1) * L.slot_bytes <= L.total,
+                                                   a.err, bounds::kRingSlot));
+            if (!ok) break;
+          }
           const unsigned char *rowp = slots + (size_t)sl * L.slot_bytes + (size_t)cq * 4 * ES;
           const int s0 = GA ? 0 : (a.g_mis0 + i * a.g_mis_k + m0 * a.g_mis_m);
           for (int r = 0; r < rows; ++r) {
@@ -536,10 +641,7 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
           st4(s.acc + (int64_t)i * ldx + col0, acc);
         } else {
           const float si = s.s[i];
-          gs.x = __fmaf_rn(si, acc.x, gs.x);
-          gs.y = __fmaf_rn(si, acc.y, gs.y);
-          gs.z = __fmaf_rn(si, acc.z, gs.z);
-          gs.w = __fmaf_rn(si, acc.w, gs.w);
+          gs = fma4(si, acc, gs);
         }
       }
       if (!ok) break;
@@ -568,7 +670,7 @@ __global__ void nb_wait_selftest_kernel(int *err, int code, long long limit_cycl
 }
 
 struct PipeTuning {
-  int T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0;
+  int T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0, x_stages = 0;
   int sm_count = 0;
 };
 
@@ -587,6 +689,7 @@ PipeTuning &tuning() {
     q.ctas_per_sm = geti("NB_PIPELINE_CTAS_PER_SM", 0);
     q.rows = geti("NB_PIPELINE_ROWS", 0);
     q.groups = geti("NB_PIPELINE_GROUPS", 0);
+    q.x_stages = geti("NB_PIPELINE_XSTAGES", 0);
 #endif
     return q;
   }();
@@ -599,7 +702,6 @@ PipeTuning &tuning() {
   return t;
 }
 
-constexpr int kSmemBudget = 227 * 1024;
 
 using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                               const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -689,23 +791,34 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   const int row_pad = rows_aligned ? 0 : 16;
   // Tile width: a box row is 256 units of T*es/256 bytes, so T is 128, 256 or 512.
   // Shapes tried in order (measured on B200, see profiles/): two CTAs per SM with two consumer
-  // groups each while the double-buffered X stage leaves room for it (K <= 16 at T = 512), else one
-  // CTA per SM with four groups; then narrower tiles.  The first shape whose ring has at least two
-  // slots per group is taken.  A tuning build's overrides replace the corresponding field of every shape.
-  struct Shape { int T, ctas, groups; };
-  const Shape shapes[] = {{512, 2, 2}, {512, 1, 4}, {256, 1, 4}, {128, 1, 4}};
-  int T = 0, ctas = 0, groups = 0, slots = 0;
+  // groups each while two X buffers leave room for it (K <= 16 at T = 512), else one CTA per SM with
+  // four groups; for K so large that two buffers of 512 columns do not fit, one buffer (the ring
+  // keeps the copies going while the next tile's models load) before narrower tiles.  The
+  // update-then-mix order first tries three X buffers, which let its averaging pass run a tile
+  // late.  The first shape whose ring has at least two slots per group is taken.  A tuning build's
+  // overrides replace the corresponding field of every shape.
+  struct Shape { int T, ctas, groups, x_stages; };
+  static const Shape mix_first_shapes[] = {{512, 2, 2, 2}, {512, 1, 4, 2}, {512, 1, 4, 1}, {256, 1, 4, 2}, {128, 1, 4, 2}};
+  static const Shape update_first_shapes[] = {{512, 1, 4, 3}, {512, 2, 2, 2}, {512, 1, 4, 2}, {512, 1, 4, 1},
+                                              {256, 1, 4, 2}, {128, 1, 4, 2}};
+  const bool mix_first = a.order == NB_ORDER_MIX_THEN_UPDATE;
+  const Shape *shapes = mix_first ? mix_first_shapes : update_first_shapes;
+  const int n_shapes = mix_first ? 5 : 6;
+  int T = 0, ctas = 0, groups = 0, slots = 0, x_stages = 0;
   bool found = false;
-  for (const Shape &sh : shapes) {
+  for (int q = 0; q < n_shapes; ++q) {
+    const Shape &sh = shapes[q];
     T = t.T ? t.T : sh.T;
     ctas = t.ctas_per_sm ? t.ctas_per_sm : sh.ctas;
     groups = t.groups ? t.groups : sh.groups;
+    x_stages = t.x_stages ? t.x_stages : sh.x_stages;
     if (T != 128 && T != 256 && T != 512) return false;
+    if (x_stages < 1 || x_stages > kMaxXStages) return false;
     if (groups > kMaxGroups) groups = kMaxGroups;
     if (groups > a.K) groups = a.K;
     while (groups > 1 && groups * (T / 4) > 512) --groups;
     if (groups < 1 || ctas < 1) return false;
-    const PipeLayout L0 = pipe_layout(a.K, T, es, R, 0, a.mix_slots, row_pad);
+    const PipeLayout L0 = pipe_layout(a.K, T, es, R, 0, a.mix_slots, row_pad, x_stages);
     const int budget = kSmemBudget / ctas - 1024;
     slots = (budget - L0.total - 256) / slot_bytes_of(T * 4, T, es, R, row_pad);
     if (t.slots && t.slots < slots) slots = t.slots;
@@ -720,8 +833,12 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   // When one item holds a learner's whole contribution (R >= M) two slots per group are enough to
   // keep the copies back to back, and deeper rings measured 1-4 % slower (MATCHA and all-reduce
   // workloads with M = 4); learners that need several items per tile use all the slots that fit.
-  if (!t.slots && R >= a.M && slots > 2 * groups) slots = 2 * groups;
-  const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots, row_pad);
+  // The update-then-mix order with its averaging pass deferred (three X buffers) releases no slot
+  // while it averages: there every slot that fits is used (cfg3 sizes: 12 slots 1.04 of the measured
+  // copy bandwidth, 8 slots 0.99).
+  const bool deferred = !mix_first && x_stages >= 3;
+  if (!t.slots && !deferred && R >= a.M && slots > 2 * groups) slots = 2 * groups;
+  const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots, row_pad, x_stages);
   if (L.total > kSmemBudget) return false;
   plan->T = T;
   plan->rows_per_item = R;
@@ -731,6 +848,7 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   plan->n_tiles = (int)cov.n_tiles;
   plan->head = (int)cov.head;
   plan->row_copies = rows_aligned ? 0 : 1;
+  plan->x_stages = x_stages;
   const int64_t max_ctas = (int64_t)ctas * t.sm_count;
   plan->grid = (int)(plan->n_tiles < max_ctas ? plan->n_tiles : max_ctas);
   return true;
@@ -765,6 +883,7 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   plan->n_tiles = (int)cov.n_tiles;
   plan->head = (int)cov.head;
   plan->row_copies = cov.rows_aligned ? 0 : 1;
+  plan->x_stages = 0;
   const int64_t max_ctas = (int64_t)ctas * t.sm_count;
   plan->grid = (int)(plan->n_tiles < max_ctas ? plan->n_tiles : max_ctas);
   return true;
@@ -793,6 +912,7 @@ void fill_pipe_args(PipeArgs *p, const StepArgs &a, const PipePlan &plan, int *e
   p->rows_per_item = plan.rows_per_item;
   p->n_tiles = plan.n_tiles;
   p->n_groups = plan.n_groups;
+  p->x_stages = plan.x_stages;
   p->err = err_flag;
 }
 }  // namespace

@@ -99,6 +99,17 @@ extern "C" int nb_step_static(int K, int64_t P, int M, float lr, float mom, floa
     a.n[i] = finished[i];
     a.s[i] = finished[i] > 0 ? 1.0f / (float)finished[i] : 0.0f;
   }
+  // extents for the bounds-checked build (there is no context, hence no error word: a failed check
+  // there only skips the access)
+  a.ext.x_lo = (uintptr_t)X;
+  a.ext.x_hi = a.ext.x_lo + sizeof(float) * (size_t)K * (size_t)ld;
+  a.ext.v_lo = (uintptr_t)V;
+  a.ext.v_hi = a.ext.v_lo + sizeof(float) * (size_t)K * (size_t)ld;
+  a.ext.acc_lo = (uintptr_t)acc;
+  a.ext.acc_hi = a.ext.acc_lo + sizeof(float) * (size_t)NB_STATIC_MAX_ELEMS;
+  a.ext.g_lo = (uintptr_t)grads;
+  a.ext.g_hi = a.ext.g_lo + (size_t)((int64_t)(K - 1) * ld_k + (int64_t)(M - 1) * ld_m + P) * (size_t)es;
+  a.err = nullptr;
   cudaStream_t st = (cudaStream_t)stream;
   // the accumulate kernel writes every element of acc[K, 0:round_up(P,4)) that the step kernel reads,
   // so nothing of the previous call's contents survives into this one

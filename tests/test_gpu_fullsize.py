@@ -36,6 +36,41 @@ def test_full_size_sampled_columns(name, steps):
     _full_size(WL.WORKLOADS[name], steps)
 
 
+def test_full_size_rows_not_16_byte_aligned():
+    """The benchmark workload with one more column: a dense stream whose rows all start at different
+    byte offsets, on the per-row bulk-copy path, in the launch configuration bench.py times."""
+    from dataclasses import replace
+    w = WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"]
+    _full_size(replace(w, P=w.P + 1, name="cfg3 with P + 1 columns"), 4, expect_row_copies=1)
+
+
+def test_mid_size_every_column():
+    """About 600 thousand columns, sixteen learners: every CTA of the persistent kernel takes several
+    tiles (stage reuse, ring phase wrap), and EVERY column is compared with the oracle."""
+    import torch
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 1200 * 512 + 24, steps=3)
+    ctx = B.context_for(w)
+    orc = H.oracle_for(w, w.P)
+    x0 = WL.init_params(w)
+    ctx.set_params(torch.from_numpy(x0).cuda())
+    orc.set_params(x0)
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        payload, values = WL.gradients_np(w, t)
+        ctx.step_fused(H.to_device(payload), n)
+        orc.step(values, n.tolist())
+        del payload, values
+    plan = ctx.get_kernel_plan()
+    assert plan["pipeline"] == 1 and plan["tiles"] == 1200 and plan["tiles"] >= 3 * plan["grid"]
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT, "X")
+    H.assert_close(ctx.get_momentum().numpy(), orc.V, H.TOL_SAME_INPUT, "V")
+    ctx.check_guards()
+    ctx.close()
+
+
 def test_more_than_two_to_the_31_columns():
     """Column indices beyond 32 bits: one learner pair, 2^31 + 1544 columns (the last window the
     oracle checks lies entirely above 2^31)."""
@@ -44,7 +79,7 @@ def test_more_than_two_to_the_31_columns():
     _full_size(w, 2)
 
 
-def _full_size(w, steps):
+def _full_size(w, steps, expect_row_copies=0):
     import torch
     from paper_2211_00889_b200.build import build_library
     build_library()
@@ -78,6 +113,8 @@ def _full_size(w, steps):
             bits, Wdev = ctx.get_device_mixing()
             assert bits == O.matcha_activation(w.seed, t, len(orc.partner), w.act_prob)
     torch.cuda.empty_cache()
+    plan = ctx.get_kernel_plan()
+    assert plan["pipeline"] == 1 and plan["row_copies"] == expect_row_copies
     X = ctx.get_params(device="cuda")[:, cols_dev].cpu().numpy()
     V = ctx.get_momentum(device="cuda")[:, cols_dev].cpu().numpy()
     ctx.check_guards()

@@ -374,7 +374,21 @@ def test_error_reporting(B):
         ctx.step_fused(g, [1, 2, -1, 1])
     with pytest.raises(B.NbError):
         ctx.step_fused(g, [1, 1, 1, 1], ld_m=50)
-    ctx.accumulate(g, [1, 1, 1, 1])
+    # the host-memory entry point validates the caller's strides before it enqueues any copy
+    gh = torch.zeros((4, 4, 100))
+    for bad in (dict(ld_m=50), dict(ld_k=150), dict(ld_m=-100), dict(ld_m=100, ld_k=-400)):
+        with pytest.raises(B.NbError) as e:
+            ctx.step_fused_host(gh, [1, 1, 1, 1], **bad)
+        assert e.value.code == B.NB_ERR_ARG
+    import ctypes
+    ones = (ctypes.c_int32 * 4)(1, 1, 1, 1)                  # a pointer that is not element-aligned
+    assert B.lib.nb_step_fused(ctx._h, g.data_ptr() + 2, B.NB_F32, 0, 0, ones, None) == B.NB_ERR_ARG
+    assert B.lib.nb_accumulate(ctx._h, g.data_ptr() + 2, B.NB_F32, 0, 0, ones, None) == B.NB_ERR_ARG
+    with pytest.raises(ValueError):
+        ctx.step_fused(g.transpose(1, 2), [1, 1, 1, 1])      # rows must be contiguous: the binding refuses
+    assert ctx.get_step() == 0                               # none of the rejected calls ran anything
+    wide = torch.zeros((4, 4, 128), device="cuda")
+    ctx.accumulate(wide[:, :, :100], [1, 1, 1, 1])           # a view with contiguous rows passes its own strides
     ctx.step()
     with pytest.raises(B.NbError):
         ctx.step()                                   # accumulator already consumed

@@ -1,5 +1,6 @@
 """nb_step_static, the entry point for callers that cannot allocate device memory, checked through
-the C ABI against the ordinary accumulate + step entry points on two iterations in a row.
+the C ABI against the ordinary accumulate + step entry points, and against the CPU oracle, on two
+iterations in a row; the second call must leave the amount of free device memory unchanged.
 
 Collected last (file name) so that a run that stops at the first failure has already run every
 other test.  It relies on nothing another test leaves behind: the library's fixed accumulator is
@@ -7,6 +8,7 @@ fully overwritten by each call before it is read."""
 import numpy as np
 import pytest
 
+from oracle import nb_oracle as O
 from paper_2211_00889_b200 import workloads as WL
 from tests import _harness as H
 
@@ -26,15 +28,26 @@ def test_static_entry_point_matches_context_path_on_two_calls_in_a_row():
         x0 = WL.init_params(w)
         ctx = B.context_for(w)                                  # the existing entry points
         ctx.set_params(torch.from_numpy(x0).cuda())
+        orc = O.Oracle(w.K, P, w.M, w.lr, w.mom, "allreduce")   # independent of both entry points
+        orc.set_params(x0)
         X = torch.zeros((w.K, ld), dtype=torch.float32, device="cuda")   # the caller's own memory
         X[:, :P] = torch.from_numpy(x0).cuda()
         V = torch.zeros_like(X)
         for t in range(2):                                      # two calls in a row share the array
             n = H.lib_counts(B, w, t)
-            g = H.to_device(WL.gradients_np(w, t)[0])
+            payload, values = WL.gradients_np(w, t)
+            g = H.to_device(payload)
             ctx.accumulate(g, n)
             ctx.step()
+            orc.step(values, n.tolist())
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             B.step_static(X, V, g, n, P, w.M, w.lr, w.mom)
+            torch.cuda.synchronize()
+            if t > 0:      # the first call on a device may load the library's code and the fixed array
+                assert torch.cuda.mem_get_info()[0] == free_before, "nb_step_static changed the free device memory"
+            H.assert_close(X[:, :P].cpu().numpy(), orc.X, H.TOL_SAME_INPUT, "X vs oracle, call %d" % t)
+            H.assert_close(V[:, :P].cpu().numpy(), orc.V, H.TOL_SAME_INPUT, "V vs oracle, call %d" % t)
             want_x, want_v = ctx.get_params(device="cuda"), ctx.get_momentum(device="cuda")
             H.assert_close(X[:, :P].cpu().numpy(), want_x.cpu().numpy(), H.TOL_SAME_INPUT, "X call %d" % t)
             H.assert_close(V[:, :P].cpu().numpy(), want_v.cpu().numpy(), H.TOL_SAME_INPUT, "V call %d" % t)
