@@ -62,6 +62,7 @@ def parse_args():
                          "nb_accumulate_minibatch per finished mini-batch, then nb_step")
     ap.add_argument("--unfused", action="store_true", help="same as --entry unfused")
     ap.add_argument("--cols", type=int, default=0, help="profiling aid: run the workload on this many columns instead of its P")
+    ap.add_argument("--learners", type=int, default=0, help="profiling aid: run the workload with this many learners instead of its K")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -632,6 +633,8 @@ def main():
     w = WL.WORKLOADS[args.workload]
     if args.cols:
         w = replace(WL.scaled(w, args.cols), name="%s[P=%d]" % (w.name, args.cols))
+    if args.learners:
+        w = replace(w, K=args.learners, name="%s[K=%d]" % (w.name, args.learners))
     if args.variant:
         topo = {"allreduce": "full", "dpsgd": "ring", "centralized": "full"}[args.variant]
         w = replace(w, variant=args.variant, topology=topo, name="%s[%s]" % (w.name, args.variant))

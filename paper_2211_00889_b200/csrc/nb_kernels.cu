@@ -4,8 +4,8 @@
 // CTA owns a contiguous column tile.  Nothing couples columns (the method only couples learners
 // and mini-batches), so CTAs never communicate, nothing waits on another CTA, and every output
 // element has exactly one writer.  All traffic is 128-bit (fp32) or 64-bit (bf16) per thread and
-// contiguous across a warp.  Gradient rows m >= n_i are never touched: skipping the abandoned
-// mini-batches is the method (Alg. 1: "break and abandon unfinished mini-batches").
+// contiguous across a warp.  Gradient rows m >= n_i are never touched: skipping the mini-batches a
+// learner had not finished when the terminal signal came is the method (Alg. 1, inner loop).
 //
 // fp32 arithmetic is written with explicit round-to-nearest intrinsics so that the fused kernel
 // and the accumulate -> step pair perform the identical operation sequence and agree bit for bit.
@@ -201,6 +201,98 @@ __global__ void __launch_bounds__(256) nb_centralized_kernel(const __grid_consta
 }
 
 // -------------------------------------------------------------------------------------------------
+// Short column ranges (the ragged tail after the bulk-copy kernel's tiles, the first tile of a stream
+// that starts off a 16-byte boundary, problems narrower than one tile).  The kernels above give a
+// thread 4 columns of ALL learners, one learner after the other: on a few hundred columns that is a
+// single CTA walking K dependent rounds of memory latency (50-100 us at K = 16-64).  Here a thread
+// owns 4 columns of ONE learner (blockDim = (column quads, K)): every learner's loads are in flight
+// at once, the learners meet in shared memory for the mix, and the range takes a few microseconds.
+// Same operations in the same order per output element: identical bits.
+//   MODE 0: sparse W   1: W = (1/K) 1 1^T   2: centralized (Alg. 3; learners folded in ascending order)
+// -------------------------------------------------------------------------------------------------
+constexpr int kTailSparse = 0, kTailMean = 1, kTailCentralized = 2;
+constexpr int kTailQuads = 16;         // column quads per CTA
+constexpr int64_t kTailMaxColumns = 4096;  // ranges up to this many columns take this kernel
+
+template <int SRC, bool ALIGNED, int MODE>
+__global__ void __launch_bounds__(kTailQuads * NB_MAX_K) nb_step_tail_kernel(const __grid_constant__ StepArgs a) {
+  extern __shared__ float4 smem[];
+  const int QC = blockDim.x, q = threadIdx.x, i = threadIdx.y, K = a.K;
+  const int tid = i * QC + q, nthreads = QC * K;
+  float4 *xs = smem;  // [K][QC]: every learner's old model (or local step, or accumulated gradient) of the CTA's columns
+  int32_t *s_col = nullptr, *s_beg = nullptr, *s_end = nullptr;
+  float *s_val = nullptr;
+  if constexpr (MODE == kTailSparse) {
+    s_col = reinterpret_cast<int32_t *>(smem + (size_t)K * QC);
+    s_val = reinterpret_cast<float *>(s_col + a.mix_slots);
+    s_beg = reinterpret_cast<int32_t *>(s_val + a.mix_slots);
+    s_end = s_beg + K;
+    for (int e = tid; e < a.mix_slots; e += nthreads) {
+      s_col[e] = a.mix->col[e];
+      s_val[e] = a.mix->val[e];
+    }
+    for (int e = tid; e < K; e += nthreads) {
+      s_beg[e] = a.mix->row_beg[e];
+      s_end[e] = a.mix->row_end[e];
+    }
+  }
+  const int64_t col0 = ((int64_t)blockIdx.x * QC + q) * kColsPerThread;
+  bool active = col0 < a.P;
+  const int nvalid = !active ? 0 : (a.P - col0 < 4) ? (int)(a.P - col0) : 4;
+  if constexpr (kDebug) {
+    if (active)
+      active = dbg_thread_footprint(a, col0, nvalid, MODE == kTailCentralized ? 1 : K, 0, SRC == kSrcAcc ? K : 0,
+                                    SRC != kSrcAcc, SRC == kSrcBF16 ? 2 : 4);
+  }
+  const int64_t row = (int64_t)i * a.ldx + col0;
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  if constexpr (MODE == kTailCentralized) {
+    xs[tid] = active ? gather<SRC, ALIGNED>(a, i, col0, nvalid) : zero;
+    __syncthreads();
+    if (active && i == 0) {
+      float4 gs = zero;
+      for (int j = 0; j < K; ++j) gs = fma4(a.s[j], xs[j * QC + q], gs);
+      const float4 v = ld4(a.V + col0);
+      const float4 x = ld4(a.X + col0);
+      const float4 vn = momentum(a.mom, v, a.inv_K, gs);
+      st4(a.V + col0, vn);
+      st4(a.X + col0, descend(x, a.lr, vn));
+    }
+  } else {
+    const bool mix_first = a.order == NB_ORDER_MIX_THEN_UPDATE;
+    float4 vn = zero;
+    if (active) {
+      const float4 x = ld4(a.X + row);
+      const float4 v = ld4(a.V + row);
+      const float4 g = gather<SRC, ALIGNED>(a, i, col0, nvalid);
+      vn = momentum(a.mom, v, a.s[i], g);
+      st4(a.V + row, vn);
+      xs[tid] = mix_first ? x : descend(x, a.lr, vn);  // Alg. 2 mixes the old models, Eq. 4-6 the local steps
+    } else {
+      xs[tid] = zero;
+    }
+    __syncthreads();
+    if (active) {
+      float4 xh;
+      if constexpr (MODE == kTailMean) {
+        xh = zero;
+        for (int j = 0; j < K; ++j) xh = add4(xh, xs[j * QC + q]);
+        xh = scale4(xh, a.inv_K);
+      } else {
+        if constexpr (kDebug) {
+          bool tab_ok = s_beg[i] >= 0 && s_beg[i] <= s_end[i] && s_end[i] <= a.mix_slots;
+          for (int e = s_beg[i]; tab_ok && e < s_end[i]; ++e) tab_ok = bounds::index_inside(s_col[e], K);
+          if (!dbg_check(tab_ok, a.err, bounds::kLearnerIndex)) return;
+        }
+        xh = mix_row(xs, QC, q, s_col, s_val, s_beg[i], s_end[i]);
+      }
+      st4(a.X + row, mix_first ? descend(xh, a.lr, vn) : xh);
+    }
+  }
+}
+
+// -------------------------------------------------------------------------------------------------
 // K3: MATCHA activation + W builder.  One Bernoulli draw per matching per step from the counter
 // generator; row i of W = I - alpha * sum_active L_j is written as (diagonal, active partners).
 // -------------------------------------------------------------------------------------------------
@@ -332,6 +424,27 @@ cudaError_t launch_accumulate_direct(const StepArgs &a, int src, cudaStream_t st
   return cudaGetLastError();
 }
 
+template <int SRC, bool ALIGNED>
+cudaError_t launch_tail_t(const StepArgs &a, int mode, cudaStream_t st) {
+  const dim3 block(kTailQuads, a.K);
+  const unsigned grid = (unsigned)((a.P + kTailQuads * kColsPerThread - 1) / (kTailQuads * kColsPerThread));
+  size_t smem = (size_t)a.K * kTailQuads * sizeof(float4);
+  if (mode == kTailSparse) {
+    smem += (size_t)a.mix_slots * 8 + (size_t)a.K * 8;
+    nb_step_tail_kernel<SRC, ALIGNED, kTailSparse><<<grid, block, smem, st>>>(a);
+  } else if (mode == kTailMean) {
+    nb_step_tail_kernel<SRC, ALIGNED, kTailMean><<<grid, block, smem, st>>>(a);
+  } else {
+    nb_step_tail_kernel<SRC, ALIGNED, kTailCentralized><<<grid, block, smem, st>>>(a);
+  }
+  return cudaGetLastError();
+}
+cudaError_t launch_tail(const StepArgs &a, int src, int mode, cudaStream_t st) {
+  if (src == kSrcAcc) return launch_tail_t<kSrcAcc, true>(a, mode, st);
+  if (src == kSrcF32) return a.g_aligned ? launch_tail_t<kSrcF32, true>(a, mode, st) : launch_tail_t<kSrcF32, false>(a, mode, st);
+  return a.g_aligned ? launch_tail_t<kSrcBF16, true>(a, mode, st) : launch_tail_t<kSrcBF16, false>(a, mode, st);
+}
+
 cudaError_t launch_step_direct(const StepArgs &a, int src, cudaStream_t st) {
   if (src == kSrcAcc) return launch_step_t<kSrcAcc, true>(a, st);
   if (src == kSrcF32) return a.g_aligned ? launch_step_t<kSrcF32, true>(a, st) : launch_step_t<kSrcF32, false>(a, st);
@@ -415,7 +528,10 @@ cudaError_t launch_step(const StepArgs &a, int src, bool pipeline, int *err_flag
   return cover_columns(
       a, p, es, planned ? &plan : nullptr, launches, used,
       [&](const StepArgs &r, const PipePlan &pl) { return launch_step_pipeline(r, es, pl, err_flag, st); },
-      [&](const StepArgs &r) { return launch_step_direct(r, src, st); });
+      [&](const StepArgs &r) {
+        if (pipeline && r.P <= kTailMaxColumns) return launch_tail(r, src, r.mean_mode ? kTailMean : kTailSparse, st);
+        return launch_step_direct(r, src, st);
+      });
 }
 
 cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, cudaStream_t st) {
@@ -426,7 +542,10 @@ cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *e
   return cover_columns(
       a, p, es, planned ? &plan : nullptr, launches, nullptr,
       [&](const StepArgs &r, const PipePlan &pl) { return launch_stream_pipeline(r, es, true, pl, err_flag, st); },
-      [&](const StepArgs &r) { return launch_centralized_direct(r, src, st); });
+      [&](const StepArgs &r) {
+        if (pipeline && r.P <= kTailMaxColumns) return launch_tail(r, src, kTailCentralized, st);
+        return launch_centralized_direct(r, src, st);
+      });
 }
 
 cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,
