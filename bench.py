@@ -38,12 +38,22 @@ UNIT = "params*learners/s"
 DEFAULT_WORKLOAD = "cfg3_dpsgd_ring_resnet50"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes per algorithmic byte, per (workload, entry): dram__bytes_read.sum + dram__bytes_write.sum
-# of the kernels of one step over the algorithmic bytes of the same step, from ncu captures of a
-# narrower column range of that workload (summarised under profiles/; traffic grows in proportion
-# to the columns).  No entry: no capture exists and `traffic` is reported as null.
+# DRAM bytes per algorithmic byte of one step, per workloads-table entry (and for the headline: the
+# entry of the same name): dram__bytes_read.sum + dram__bytes_write.sum of all kernels of a step
+# over the algorithmic bytes of that step, from ncu captures of a narrower column range of the same
+# workload (profiles/dram_traffic_per_workload_and_entry.md; traffic grows in proportion to the
+# columns).  No entry: no capture exists and `traffic` is reported as null.
 TRAFFIC_PER_ALGORITHMIC_BYTE = {
-    ("cfg3_dpsgd_ring_resnet50", "nb_step_fused"): 0.988,
+    "cfg3_dpsgd_ring_resnet50": 0.988,
+    "cfg3_dpsgd_ring_resnet50[P+1, rows not 16-byte aligned]": 0.988,
+    "cfg3_dpsgd_ring_resnet50[update_then_mix]": 0.987,
+    "cfg3_dpsgd_ring_resnet50[unfused]": 1.284,
+    "cfg3_dpsgd_ring_resnet50[centralized]": 0.997,
+    "cfg2_allreduce_resnet18": 0.990,
+    "cfg4_matcha_vgg16": 0.980,
+    "cfg5_scale_allreduce": 0.990,
+    "cfg5_scale_ring": 0.990,
+    "ring_K64_P12.8M": 0.987,
 }
 
 
@@ -61,6 +71,8 @@ def parse_args():
                     help="fused: nb_step_fused; unfused: nb_accumulate + nb_step; streaming: one "
                          "nb_accumulate_minibatch per finished mini-batch, then nb_step")
     ap.add_argument("--unfused", action="store_true", help="same as --entry unfused")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "direct"],
+                    help="direct: the direct-load kernels only (NB_OPT_KERNEL), for comparison with the bulk-copy pipeline")
     ap.add_argument("--cols", type=int, default=0, help="profiling aid: run the workload on this many columns instead of its P")
     ap.add_argument("--learners", type=int, default=0, help="profiling aid: run the workload with this many learners instead of its K")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -249,7 +261,8 @@ def run_reference(args, w):
 class Runner:
     """One workload resident on the device: context, gradient buffers, and the timed loop."""
 
-    def __init__(self, B, WL, w, dev, order="mix_then_update", seed_offset=0, bufs=None, row_shift=0, pitch=0):
+    def __init__(self, B, WL, w, dev, order="mix_then_update", seed_offset=0, bufs=None, row_shift=0, pitch=0,
+                 kernel="auto"):
         import torch
         self.B, self.WL, self.w, self.dev, self.torch = B, WL, w, dev, torch
         self.es = 4 if w.grad_dtype == "f32" else 2
@@ -282,6 +295,8 @@ class Runner:
         self.ctx.set_params(x0)
         if order == "update_then_mix":
             self.ctx.set_option(B.NB_OPT_ORDER, B.NB_ORDER_UPDATE_THEN_MIX)
+        if kernel == "direct":
+            self.ctx.set_option(B.NB_OPT_KERNEL, B.NB_KERNEL_DIRECT)
         self.order = order
 
     def counts(self, t):
@@ -370,8 +385,7 @@ def table_entry(label, w, order, entry, r, peak, steps, note=None):
     ms = r["total_ms"] / steps
     achieved = alg / (r["launch_ms"] * 1e-3) / 1e9
     moved = r["own_bytes_per_step"] / (r["launch_ms"] * 1e-3) / 1e9
-    tr = TRAFFIC_PER_ALGORITHMIC_BYTE.get((w.name, ENTRY_NAMES[entry] if order == "mix_then_update"
-                                           else ENTRY_NAMES[entry] + "[update_then_mix]"))
+    tr = TRAFFIC_PER_ALGORITHMIC_BYTE.get(label)
     out = {"name": label, "K": w.K, "P": w.P, "M": w.M, "grad_dtype": w.grad_dtype, "variant": w.variant,
            "topology": w.topology, "order": order, "entry": ENTRY_NAMES[entry], "steps": steps,
            "ms_per_step": ms, "step_ms_device": r["launch_ms"], "value": w.K * w.P / (ms * 1e-3), "unit": UNIT,
@@ -478,7 +492,7 @@ def run_ours(args, w):
             print("[bench] " + msg, file=sys.stderr, flush=True)
 
     # rank r owns columns [r*P, (r+1)*P) of an N*P-wide problem: same counts everywhere, own data
-    runner = Runner(B, WL, w, dev, order=args.order, seed_offset=1000 * rank)
+    runner = Runner(B, WL, w, dev, order=args.order, seed_offset=1000 * rank, kernel=args.kernel)
     es = runner.es
     if world > 1:   # every rank derives the counts by itself; they must coincide (checked outside the timed region)
         assert sharding.counts_agree(runner.counts(args.warmup), dev), "ranks disagree on the finished counts"
@@ -491,12 +505,21 @@ def run_ours(args, w):
     peak, peak_kind = measured_peak()
     bytes_per_launch = sum(r["alg_bytes"]) / args.steps
     achieved = bytes_per_launch / (r["launch_ms"] * 1e-3) / 1e9
-    tr = TRAFFIC_PER_ALGORITHMIC_BYTE.get((w.name.split("[")[0], ENTRY_NAMES[args.entry]
-                                           if args.order == "mix_then_update" and not args.variant else ""))
+    head_label = w.name
+    if args.kernel != "auto" or args.cols or args.learners:
+        head_label = None                                  # not a captured configuration
+    elif args.variant:
+        head_label = None if args.variant != "centralized" or args.entry != "fused" else w.name
+    elif args.entry != "fused":
+        head_label = "%s[%s]" % (w.name, args.entry)
+    elif args.order != "mix_then_update":
+        head_label = "%s[%s]" % (w.name, args.order)
+    tr = TRAFFIC_PER_ALGORITHMIC_BYTE.get(head_label)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": tr * bytes_per_launch if tr else None,
                 "peak_source": "of " + peak_kind,
-                "kernel": "nb_step_pipeline_kernel (fused accumulate+mix+momentum+update)" if args.entry == "fused"
+                "kernel": ("nb_step_kernel (direct loads; fused accumulate+mix+momentum+update)" if args.kernel == "direct"
+                           else "nb_step_pipeline_kernel (fused accumulate+mix+momentum+update)") if args.entry == "fused"
                           else ENTRY_NAMES[args.entry],
                 "algorithmic_bytes_per_launch": bytes_per_launch, "launch_ms": r["launch_ms"],
                 "frac_of_8TBps_nominal": achieved / 8000.0, "mean_sum_finished": r["mean_sum_finished"],
