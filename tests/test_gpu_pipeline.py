@@ -251,6 +251,42 @@ def test_accumulate_on_pipeline_sizes(B, dtype, M):
     a.close(); b.close(); d.close()
 
 
+@pytest.mark.parametrize("K", [1, 2, 5, 31, 64])
+@pytest.mark.parametrize("variant,order", [("dpsgd", 0), ("dpsgd", 1), ("allreduce", 0), ("allreduce", 1),
+                                           ("centralized", 0)])   # one shared model has no mixing order
+def test_short_range_kernel_agrees_with_the_direct_kernel_bitwise(B, K, variant, order):
+    """Column ranges of a few hundred columns (ragged tails, problems narrower than a tile) run on the
+    learner-parallel kernel (a thread owns one learner's 4 columns); NB_KERNEL_DIRECT runs the same
+    problem on the column-per-thread kernel.  Same bits, any learner count up to NB_MAX_K, both
+    orders, all mixing modes, aligned and unaligned rows, fused and unfused."""
+    import torch
+    for P, dtype in ((300, "bf16"), (515, "f32"), (7, "bf16"), (512 + 129, "bf16")):
+        rng = np.random.default_rng(1000 * K + P)
+        M = 5
+        topo = B.make_topology("ring") if variant == "dpsgd" else None
+        ctxs = [B.NbContext(K, P, M, 0.05, 0.9, variant, topo) for _ in range(3)]
+        a, u, d = ctxs                                   # fused, unfused, direct kernels only
+        d.set_option(B.NB_OPT_KERNEL, B.NB_KERNEL_DIRECT)
+        x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+        for c in ctxs:
+            if variant != "centralized":
+                c.set_option(B.NB_OPT_ORDER, order)
+            c.set_params(torch.from_numpy(x0).cuda())
+        tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+        for t in range(3):
+            G = (torch.from_numpy(rng.standard_normal((K, M, P)).astype(np.float32)) * 0.01).to(tdt).cuda()
+            n = rng.integers(0, M + 1, K)
+            a.step_fused(G, n)
+            u.accumulate(G, n); u.step()
+            d.step_fused(G, n)
+            assert d.get_kernel_plan()["pipeline"] == 0
+        for c in (u, d):
+            assert torch.equal(a.get_params(), c.get_params()) and torch.equal(a.get_momentum(), c.get_momentum())
+        for c in ctxs:
+            c.check_guards()
+            c.close()
+
+
 def test_aligned_and_unaligned_streams_interleave(B):
     """A context may see aligned streams (box copies) and unaligned ones (per-row bulk copies plus a
     first tile on the direct-load kernel) in any order; state and results must be those of a context
