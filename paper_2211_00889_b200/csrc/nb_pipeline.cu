@@ -405,6 +405,11 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
       // X buffers the averaging pass of tile t runs after the first pass of tile t+1: the groups
       // reach the rendezvous with a tile of slack and nobody idles at it.
       const bool defer = !mix_first && NXS >= 3;
+      // With two buffers the averaging pass of tile t-1 runs in the MIDDLE of tile t's first pass (after
+      // half of this group's learners): half a pass of slack at the rendezvous, and the buffer it frees
+      // still has the other half of the pass to receive tile t+1's models.
+      const bool defer_half = !mix_first && NXS == 2;
+      const int half_at = ((K - grp + NG - 1) / NG) / 2;  // learners of this group done before the late pass
 
       // Second pass of update-then-mix on buffer ub (columns at ucol0): x_i = sum_j W_ij y_j.
       auto average_and_store = [&](int ub, uint32_t upar, int64_t ucol0) -> bool {
@@ -454,7 +459,11 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
           for (int j = 0; j < K; ++j) mean = add4(mean, xs4[j * nq + cq]);
           mean = scale4(mean, s.inv_K);
         }
-        for (int i = grp; ok && i < K; i += NG) {  // this group's learners, from its own ring
+        int done = 0;
+        for (int i = grp; ok && i < K; i += NG, ++done) {  // this group's learners, from its own ring
+          if (defer_half && titer > 0 && done == half_at) {
+            if (!(ok = average_and_store(prev_xb, prev_xpar, prev_col0))) break;
+          }
           const int n = s.n[i];
           float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
           float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -498,10 +507,10 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
           // this group's y of the tile are staged: tell the others (bounded mbarrier rendezvous)
           __syncwarp();
           if (lane == 0) mbar_arrive(&ybar[xb]);
-          if (!defer) {
+          if (defer) {
+            if (titer > 0 && !(ok = average_and_store(prev_xb, prev_xpar, prev_col0))) break;
+          } else if (!defer_half) {
             if (!(ok = average_and_store(xb, xpar, col0))) break;
-          } else if (titer > 0) {
-            if (!(ok = average_and_store(prev_xb, prev_xpar, prev_col0))) break;
           }
           prev_xb = xb;
           prev_xpar = xpar;
@@ -509,7 +518,7 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
         }
         if (++xb == NXS) { xb = 0; xpar ^= 1; }
       }
-      if (ok && defer && titer > 0) ok = average_and_store(prev_xb, prev_xpar, prev_col0);  // the last tile's second pass
+      if (ok && (defer || defer_half) && titer > 0) ok = average_and_store(prev_xb, prev_xpar, prev_col0);  // the last tile's second pass
     }
   }
   if (!ok) drain_and_exit_delay();
