@@ -792,10 +792,10 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   PipeTuning &t = tuning();
   if ((uintptr_t)a.G % es != 0) return false;
   if (!encode_fn()) return false;
-  int R = t.rows ? t.rows : 8;
-  if (R < 1) R = 1;
-  if (R > kMaxRowsPerItem) R = kMaxRowsPerItem;
-  if (R > a.M) R = a.M;
+  int Rmax = t.rows ? t.rows : 8;
+  if (Rmax < 1) Rmax = 1;
+  if (Rmax > kMaxRowsPerItem) Rmax = kMaxRowsPerItem;
+  if (Rmax > a.M) Rmax = a.M;
   const bool rows_aligned = coverage(a, es, 512).rows_aligned;
   const int row_pad = rows_aligned ? 0 : 16;
   // Tile width: a box row is 256 units of T*es/256 bytes, so T is 128, 256 or 512.
@@ -804,19 +804,23 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   // four groups; for K so large that two buffers of 512 columns do not fit, one buffer (the ring
   // keeps the copies going while the next tile's models load) before narrower tiles.  The
   // update-then-mix order first tries three X buffers, which let its averaging pass run a tile
-  // late.  The first shape whose ring has at least two slots per group is taken.  A tuning build's
-  // overrides replace the corresponding field of every shape.
-  struct Shape { int T, ctas, groups, x_stages; };
-  static const Shape mix_first_shapes[] = {{512, 2, 2, 2}, {512, 1, 4, 2}, {512, 1, 4, 1}, {256, 1, 4, 2}, {128, 1, 4, 2}};
-  static const Shape update_first_shapes[] = {{512, 1, 4, 3}, {512, 2, 2, 2}, {512, 1, 4, 2}, {512, 1, 4, 1},
-                                              {256, 1, 4, 2}, {128, 1, 4, 2}};
+  // late.  The first shape whose ring has at least two slots per group is taken; a shape with rows = 4
+  // halves the rows per ring item (the slots shrink) so that 512-column tiles still fit where 8-row
+  // items do not (K = 64 with fp32 gradients: 0.94 on 256-column tiles).  A tuning build's overrides
+  // replace the corresponding field of every shape.
+  struct Shape { int T, ctas, groups, x_stages, rows; };
+  static const Shape mix_first_shapes[] = {{512, 2, 2, 2, 8}, {512, 1, 4, 2, 8}, {512, 1, 4, 1, 8}, {512, 1, 4, 1, 4},
+                                           {256, 1, 4, 2, 8}, {128, 1, 4, 2, 8}};
+  static const Shape update_first_shapes[] = {{512, 1, 4, 3, 8}, {512, 2, 2, 2, 8}, {512, 1, 4, 2, 8}, {512, 1, 4, 1, 8},
+                                              {512, 1, 4, 1, 4}, {256, 1, 4, 2, 8}, {128, 1, 4, 2, 8}};
   const bool mix_first = a.order == NB_ORDER_MIX_THEN_UPDATE;
   const Shape *shapes = mix_first ? mix_first_shapes : update_first_shapes;
-  const int n_shapes = mix_first ? 5 : 6;
-  int T = 0, ctas = 0, groups = 0, slots = 0, x_stages = 0;
+  const int n_shapes = mix_first ? 6 : 7;
+  int T = 0, ctas = 0, groups = 0, slots = 0, x_stages = 0, R = Rmax;
   bool found = false;
   for (int q = 0; q < n_shapes; ++q) {
     const Shape &sh = shapes[q];
+    R = sh.rows < Rmax ? sh.rows : Rmax;
     T = t.T ? t.T : sh.T;
     ctas = t.ctas_per_sm ? t.ctas_per_sm : sh.ctas;
     groups = t.groups ? t.groups : sh.groups;
