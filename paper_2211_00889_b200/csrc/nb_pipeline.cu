@@ -843,14 +843,15 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   const Coverage cov = coverage(a, es, T);
   if (cov.n_tiles < 1) return false;
   if ((cov.n_tiles + 1) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
-  // When one item holds a learner's whole contribution (R >= M) two slots per group are enough to
-  // keep the copies back to back, and deeper rings measured 1-4 % slower (MATCHA and all-reduce
-  // workloads with M = 4); learners that need several items per tile use all the slots that fit.
-  // The update-then-mix order with its averaging pass deferred (three X buffers) releases no slot
-  // while it averages: there every slot that fits is used (cfg3 sizes: 12 slots 1.04 of the measured
-  // copy bandwidth, 8 slots 0.99).
-  const bool deferred = !mix_first && x_stages >= 3;
-  if (!t.slots && !deferred && R >= a.M && slots > 2 * groups) slots = 2 * groups;
+  // Ring depth.  With two X buffers in the Alg. 2 order, when one item holds a learner's whole
+  // contribution (R >= M) two slots per group keep the copies back to back and deeper rings measured
+  // 1-4 % slower (more copies in flight than the latency needs only spread the chip over more DRAM
+  // rows at once); learners that need several items per tile use all the slots that fit.  Every slot
+  // that fits is also used by the shapes whose consumers pause: the single X buffer of K > 32 (the ring
+  // is what keeps memory busy while the next tile's models load: K = 40 / 48, 12 slots 1.03 of the
+  // measured copy bandwidth, 8 slots 0.98) and the update-then-mix order (no slot is released while a
+  // group averages: cfg3 sizes 12 slots 1.04, 8 slots 0.99).
+  if (!t.slots && mix_first && x_stages == 2 && R >= a.M && slots > 2 * groups) slots = 2 * groups;
   const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots, row_pad, x_stages);
   if (L.total > kSmemBudget) return false;
   plan->T = T;
