@@ -9,9 +9,11 @@
 // issue-bound):
 //
 //   * the CTA owns column tiles of T columns (persistent, tile = blockIdx.x + k * gridDim.x);
-//   * an X producer thread brings the K old model rows X[:, tile] into a double-buffered X stage
-//     with one box copy per tile (the mix needs every neighbour's OLD value while X is updated in
-//     place); tile t+1's models load while tile t is consumed;
+//   * an X producer thread brings the K old model rows X[:, tile] into the X stage with one box copy
+//     per tile (the mix needs every neighbour's OLD value while X is updated in place).  The stage
+//     has two buffers, so tile t+1's models load while tile t is consumed; one buffer where two do
+//     not fit (K > 32: the ring keeps the copies going meanwhile); three for the update-then-mix
+//     order (Eq. 4-6), whose averaging pass then runs one tile late;
 //   * the consumers form NG groups of T/4 threads; group g owns the learners i = g, g+NG, ...
 //     (their updates are independent once the old models are staged) and a PRIVATE ring of slots;
 //     its own producer thread streams that group's "items" into the ring: item = momentum row
