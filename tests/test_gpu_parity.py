@@ -105,6 +105,17 @@ def test_configs_scaled_columns(B, name, P, fused):
     _run(B, w, w.steps, fused=fused, check_steps=(10,), with_unrounded=(w.grad_dtype == "bf16"))
 
 
+@pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16",
+                                  "cfg5_scale_allreduce", "cfg5_scale_ring"])
+def test_configs_for_their_full_number_of_steps(B, name):
+    """Every configuration for as many steps as it names (50, 50, 20, 20, 20), on a column range of a
+    few tiles: the tolerance holds after 10 steps (where the contract states it) and still at the end."""
+    w = WL.scaled(WL.WORKLOADS[name], 2 * 1024 + 72)
+    assert w.steps in (20, 50)
+    errs = _run(B, w, w.steps, fused=True, check_steps=(10, w.steps), with_unrounded=(w.grad_dtype == "bf16"))
+    assert set(errs) == {10, w.steps}
+
+
 @pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16"])
 @pytest.mark.parametrize("P", [1, 3, 7, 4099, 1025])
 def test_ragged_and_unaligned_sizes(B, name, P):
