@@ -98,3 +98,62 @@ def test_random_configuration(case_id):
         H.assert_close(V, v_ps, H.TOL_SAME_INPUT, str(c))
     ctx.check_guards()
     ctx.close()
+
+
+@pytest.mark.parametrize("case_id", range(60))
+def test_random_differential_between_kernel_families(case_id):
+    """The same random problem through the default kernels (bulk-copy pipeline in whichever shape the
+    planner picks - box or per-row copies, one to three X buffers, either mixing order - plus the
+    short-range kernel on what is left) and through the direct-load kernels alone: identical bits.
+    Learner counts up to NB_MAX_K, streams shifted off their 16-byte boundary, padded rows."""
+    import torch
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    rng = np.random.default_rng(9000 + case_id)
+    variant = str(rng.choice(["allreduce", "ring", "matcha", "centralized"]))
+    K = int(rng.choice([1, 2, 3, 7, 16, 17, 25, 33, 48, 64])) if variant != "matcha" else int(rng.choice([4, 8, 16, 24]))
+    M = int(rng.integers(1, 21))
+    P = int(rng.choice([rng.integers(1, 512), 512 * rng.integers(1, 10), 512 * rng.integers(1, 10) + rng.integers(1, 512)]))
+    dtype = torch.bfloat16 if rng.integers(0, 2) else torch.float32
+    order = int(rng.integers(0, 2))
+    shift = int(rng.choice([0, 0, 1, 3]))
+    pad = int(rng.choice([0, 0, 8, 5]))
+    fused = bool(rng.integers(0, 2))
+    seed = int(rng.integers(0, 2 ** 40))
+
+    def make():
+        if variant == "allreduce":
+            return B.NbContext(K, P, M, 0.05, 0.9, "allreduce")
+        if variant == "ring":
+            return B.NbContext(K, P, M, 0.05, 0.9, "dpsgd", B.make_topology("ring"))
+        if variant == "matcha":
+            topo = B.make_topology("random_regular", degree=3 if K > 4 else 2, seed=seed, alpha=0.2, act_prob=0.6)
+            return B.NbContext(K, P, M, 0.05, 0.9, "matcha", topo)
+        return B.NbContext(K, P, M, 0.05, 0.9, "centralized")
+
+    a, d = make(), make()
+    d.set_option(B.NB_OPT_KERNEL, B.NB_KERNEL_DIRECT)
+    x0 = torch.from_numpy((rng.standard_normal(P) * 0.01).astype(np.float32)).cuda()
+    for c in (a, d):
+        if variant != "centralized":
+            c.set_option(B.NB_OPT_ORDER, order)
+        c.set_params(x0)
+    for t in range(2):
+        G = (torch.from_numpy(rng.standard_normal((K, M, P)).astype(np.float32)) * 0.01).to(dtype).cuda()
+        flat = torch.zeros(K * M * (P + pad) + shift, dtype=dtype, device="cuda")
+        g = flat[shift:].view(K, M, P + pad)[:, :, :P]          # rows P + pad apart, `shift` elements off the allocation
+        g.copy_(G)
+        n = rng.integers(0, M + 1, K)
+        for c in (a, d):
+            if fused:
+                c.step_fused(g, n)
+            else:
+                c.accumulate(g, n)
+                c.step()
+    case = dict(variant=variant, K=K, M=M, P=P, dtype=str(dtype), order=order, shift=shift, pad=pad, fused=fused,
+                plan=a.get_kernel_plan())
+    assert torch.equal(a.get_params(), d.get_params()), case
+    assert torch.equal(a.get_momentum(), d.get_momentum()), case
+    a.check_guards(); d.check_guards()
+    a.close(); d.close()
