@@ -67,7 +67,7 @@ def parse_args():
     ap.add_argument("--variant", default="", choices=["", "allreduce", "dpsgd", "centralized"],
                     help="run the workload's sizes with another variant (dpsgd = ring)")
     ap.add_argument("--order", default="mix_then_update", choices=["mix_then_update", "update_then_mix"])
-    ap.add_argument("--entry", default="fused", choices=["fused", "unfused", "streaming"],
+    ap.add_argument("--entry", default="fused", choices=["fused", "unfused", "streaming", "streaming_hold"],
                     help="fused: nb_step_fused; unfused: nb_accumulate + nb_step; streaming: one "
                          "nb_accumulate_minibatch per finished mini-batch, then nb_step")
     ap.add_argument("--unfused", action="store_true", help="same as --entry unfused")
@@ -107,7 +107,8 @@ def host_threads():
 
 
 ENTRY_NAMES = {"fused": "nb_step_fused", "unfused": "nb_accumulate+nb_step",
-               "streaming": "nb_accumulate_minibatch x sum(n_i) + nb_step"}
+               "streaming": "nb_accumulate_minibatch x sum(n_i) + nb_step",
+               "streaming_hold": "nb_accumulate_minibatch x sum(n_i) [NB_STREAMING_HOLD] + nb_step"}
 
 
 def config_of(w, order, entry, world):
@@ -313,6 +314,9 @@ class Runner:
         else:
             # Alg. 1 inner loop as the gradients arrive: round m delivers mini-batch m of every learner
             # that finished it; the fastest learner's M-th delivery raises the terminal signal last
+            if entry == "streaming_hold" and not getattr(self, "_hold_set", False):
+                ctx.set_option(self.B.NB_OPT_STREAMING, self.B.NB_STREAMING_HOLD)
+                self._hold_set = True
             ctx.begin_iteration()
             for m in range(self.w.M):
                 for i in range(self.w.K):
@@ -460,6 +464,9 @@ def other_workloads(args, B, WL, dev, base_runner, peak, local, log):
     run(w3.name + "[streaming]", w3, entry="streaming", bufs=shared,
         note="Alg. 1 inner loop as the gradients arrive: one launch per finished mini-batch, accumulator "
              "read-modify-write per delivery")
+    run(w3.name + "[streaming_hold]", w3, entry="streaming_hold", bufs=shared,
+        note="the same deliveries only recorded (NB_STREAMING_HOLD): nb_step runs the fused step on the delivered "
+             "vectors where they lie, one bulk copy per row from a table of row pointers")
     return out, shared
 
 

@@ -16,7 +16,8 @@ NB_OK, NB_ERR_ARG, NB_ERR_STATE, NB_ERR_CUDA, NB_ERR_NOMEM, NB_ERR_UNSUPPORTED =
 NB_ALLREDUCE, NB_DPSGD, NB_MATCHA, NB_CENTRALIZED = 0, 1, 2, 3
 NB_F32, NB_BF16 = 0, 1
 NB_TOPO_FULL, NB_TOPO_RING, NB_TOPO_CSR, NB_TOPO_MATCHINGS, NB_TOPO_RANDOM_REGULAR = 0, 1, 2, 3, 4
-NB_OPT_NORM, NB_OPT_ORDER, NB_OPT_KERNEL = 0, 1, 2
+NB_OPT_NORM, NB_OPT_ORDER, NB_OPT_KERNEL, NB_OPT_STREAMING = 0, 1, 2, 3
+NB_STREAMING_ACCUMULATE, NB_STREAMING_HOLD = 0, 1
 NB_KERNEL_AUTO, NB_KERNEL_DIRECT = 0, 1
 NB_NORM_MEAN, NB_NORM_PAPER = 0, 1
 NB_ORDER_MIX_THEN_UPDATE, NB_ORDER_UPDATE_THEN_MIX = 0, 1

@@ -8,6 +8,7 @@
 #include <new>
 #include <utility>
 #include <string>
+#include <vector>
 
 #include "nb_internal.h"
 #include "nb_kernels.h"
@@ -37,6 +38,11 @@ struct nb_ctx {
   bool acc_fresh = false, device_mix_valid = false;
   int32_t n_acc[NB_MAX_K] = {0};
   bool streaming = false, terminal = false;  // nb_begin_iteration / nb_accumulate_minibatch state
+  int streaming_mode = NB_STREAMING_ACCUMULATE;
+  bool holding = false;                      // this iteration's deliveries were recorded, not accumulated
+  int hold_dtype = NB_F32;
+  std::vector<const void *> h_rows;          // [K*M] row pointers of the held deliveries (host mirror)
+  const void **d_rows = nullptr;             // the same table on the device
   int acc_esize = 4;
   int64_t sum_finished = 0, launches = 0;
   double alg_bytes = 0.0;
@@ -350,6 +356,7 @@ int nb_destroy(nb_ctx *c) {
   cudaFree(c->d_mix);
   cudaFree(c->d_partner);
   cudaFree(c->d_err);
+  cudaFree(c->d_rows);
   cudaFree(c->staging);
   if (c->s_copy) cudaStreamDestroy(c->s_copy);
   if (c->s_out) cudaStreamDestroy(c->s_out);
@@ -373,6 +380,12 @@ int nb_set_option(nb_ctx *c, int key, int64_t value) {
   if (key == NB_OPT_ORDER) {
     if (value != NB_ORDER_MIX_THEN_UPDATE && value != NB_ORDER_UPDATE_THEN_MIX) return fail(c, NB_ERR_ARG, "unknown order");
     c->order = (int)value;
+    return NB_OK;
+  }
+  if (key == NB_OPT_STREAMING) {
+    if (value != NB_STREAMING_ACCUMULATE && value != NB_STREAMING_HOLD) return fail(c, NB_ERR_ARG, "unknown streaming mode");
+    if (c->streaming) return fail(c, NB_ERR_STATE, "the streaming mode cannot change inside an iteration");
+    c->streaming_mode = (int)value;
     return NB_OK;
   }
   if (key == NB_OPT_KERNEL) {
@@ -436,6 +449,11 @@ int nb_begin_iteration(nb_ctx *c) {
   c->terminal = false;
   c->acc_fresh = true;
   c->acc_esize = 4;
+  c->holding = c->streaming_mode == NB_STREAMING_HOLD;
+  if (c->holding) {
+    c->h_rows.assign((size_t)c->K * (size_t)c->M, nullptr);
+    if (!c->d_rows) NB_CUDA(c, cudaMalloc(&c->d_rows, sizeof(void *) * (size_t)c->K * (size_t)c->M));
+  }
   return NB_OK;
 }
 
@@ -449,6 +467,17 @@ int nb_accumulate_minibatch(nb_ctx *c, int learner, const void *grad, int dtype,
   const int es = dtype == NB_F32 ? 4 : 2;
   const bool aligned = (uintptr_t)grad % (size_t)(4 * es) == 0;
   if ((uintptr_t)grad % (size_t)es != 0) return fail(c, NB_ERR_ARG, "grad is not aligned to its element size");
+  if (c->holding) {  // record the vector; nb_step reads it in place
+    if ((uintptr_t)grad % 16 != 0) return fail(c, NB_ERR_ARG, "NB_STREAMING_HOLD needs 16-byte aligned gradient vectors");
+    bool first = true;
+    for (int i = 0; i < c->K; ++i) first = first && c->n_acc[i] == 0;
+    if (first) c->hold_dtype = dtype;
+    else if (dtype != c->hold_dtype) return fail(c, NB_ERR_ARG, "NB_STREAMING_HOLD needs one dtype per iteration");
+    c->h_rows[(size_t)learner * (size_t)c->M + (size_t)c->n_acc[learner]] = grad;
+    c->acc_esize = es;
+    if (++c->n_acc[learner] == c->M) c->terminal = true;
+    return NB_OK;
+  }
   NB_CUDA(c, nb::launch_add_minibatch(c->acc + (int64_t)learner * c->ldx, grad, dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16,
                                       aligned, c->P, c->n_acc[learner] == 0, extents_of(c, nullptr, 0, 0, es), c->d_err,
                                       (cudaStream_t)stream));
@@ -468,12 +497,6 @@ int nb_get_finished(const nb_ctx *c, int32_t *finished, int32_t *terminal) {
 int nb_step(nb_ctx *c, void *stream) {
   NB_ENTER(c);
   if (!c->acc_fresh) return fail(c, NB_ERR_STATE, "nb_step needs an nb_accumulate since the last step");
-  if (c->streaming) {  // learners that delivered nothing contribute a zero accumulator
-    for (int i = 0; i < c->K; ++i)
-      if (c->n_acc[i] == 0)
-        NB_CUDA(c, cudaMemsetAsync(c->acc + (int64_t)i * c->ldx, 0, sizeof(float) * (size_t)c->ldx, (cudaStream_t)stream));
-    c->streaming = false;
-  }
   nb::StepArgs a;
   std::memset(&a, 0, sizeof(a));
   a.X = c->X;
@@ -489,6 +512,22 @@ int nb_step(nb_ctx *c, void *stream) {
   a.err = c->d_err;
   std::memcpy(a.n, c->n_acc, sizeof(a.n));
   record_stats(c, a, c->acc_esize);
+  if (c->streaming && c->holding) {
+    // the recorded vectors are the gradient stream: the fused step reads them where they lie
+    NB_CUDA(c, cudaMemcpyAsync(c->d_rows, c->h_rows.data(), sizeof(void *) * c->h_rows.size(), cudaMemcpyHostToDevice,
+                               (cudaStream_t)stream));
+    c->streaming = false;
+    c->holding = false;
+    a.row_ptrs = c->d_rows;
+    // (g_aligned stays 1: the vectors are 16-byte aligned and every thread starts at a multiple of 4 columns)
+    return run_update(c, &a, c->hold_dtype == NB_F32 ? nb::kSrcF32 : nb::kSrcBF16, (cudaStream_t)stream);
+  }
+  if (c->streaming) {  // learners that delivered nothing contribute a zero accumulator
+    for (int i = 0; i < c->K; ++i)
+      if (c->n_acc[i] == 0)
+        NB_CUDA(c, cudaMemsetAsync(c->acc + (int64_t)i * c->ldx, 0, sizeof(float) * (size_t)c->ldx, (cudaStream_t)stream));
+    c->streaming = false;
+  }
   return run_update(c, &a, nb::kSrcAcc, (cudaStream_t)stream);
 }
 

@@ -47,7 +47,7 @@ __device__ __forceinline__ bool dbg_thread_footprint(const StepArgs &a, int64_t 
                           dbg_rows_inside(a.acc + (int64_t)acc_row0 * a.ldx, a.ldx, acc_rows, col0, 4, 4, a.ext.acc_lo,
                                           a.ext.acc_hi),
                       a.err, bounds::kStateAddress);
-  if (reads_g) {
+  if (reads_g && !a.row_ptrs) {  // held rows are vectors of P elements of their own: col0 < P is the whole check
     const unsigned char *g = reinterpret_cast<const unsigned char *>(a.G);
     const unsigned char *last = g + ((int64_t)(a.K - 1) * a.ld_k + (int64_t)(a.M - 1) * a.ld_m) * g_esize;
     ok = dbg_check(dbg_rows_inside(g, 0, 1, col0, nvalid, g_esize, a.ext.g_lo, a.ext.g_hi) &&

@@ -34,13 +34,17 @@ __device__ __forceinline__ float4 gather(const StepArgs &a, int i, int64_t col0,
   } else {
     using E = typename ElemOf<SRC>::type;
     const E *base = reinterpret_cast<const E *>(a.G) + (int64_t)i * a.ld_k + col0;
+    const void *const *rows = a.row_ptrs ? a.row_ptrs + (int64_t)i * a.M : nullptr;  // held rows: one vector per row
     const int n = a.n[i];
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int m0 = 0; m0 < n; m0 += kChunk) {
       Raw<SRC> r[kChunk];
 #pragma unroll
       for (int u = 0; u < kChunk; ++u)
-        if (m0 + u < n) r[u] = load_raw<ALIGNED>(base + (int64_t)(m0 + u) * a.ld_m, nvalid, (Raw<SRC> *)nullptr);
+        if (m0 + u < n) {
+          const E *row = rows ? reinterpret_cast<const E *>(rows[m0 + u]) + a.row_col0 + col0 : base + (int64_t)(m0 + u) * a.ld_m;
+          r[u] = load_raw<ALIGNED>(row, nvalid, (Raw<SRC> *)nullptr);
+        }
 #pragma unroll
       for (int u = 0; u < kChunk; ++u)
         if (m0 + u < n) {
@@ -400,6 +404,7 @@ StepArgs acc_as_stream(const StepArgs &a) {
 
 StepArgs column_range(const StepArgs &a, int64_t c0, int64_t cols, int es) {
   StepArgs r = a;
+  r.row_col0 += c0;  // held rows: the table stays as it is, the kernels add the range's first column
   r.X += c0;
   r.V += c0;
   r.acc += c0;

@@ -29,8 +29,10 @@ struct StepArgs {
   float *V;            // [K, ldx] momentum
   float *acc;          // [K, ldx] accumulator (written by accumulate, read by the unfused step)
   const void *G;       // gradient stream, element (i,m,p) at G[i*ld_k + m*ld_m + p]
+  const void *const *row_ptrs;  // or (G == NULL): device table [K*M], row (i,m) is the vector row_ptrs[i*M+m][0..P)
   const MixTable *mix; // sparse W (ignored in mean mode)
   int64_t ldx, ld_m, ld_k, P;
+  int64_t row_col0;    // row_ptrs only: the first column of this launch's range inside the held vectors
   int32_t K, M;
   int32_t mix_slots;   // number of table slots to stage in shared memory
   int32_t mean_mode;   // 1: W = (1/K) 1 1^T, computed as one column mean
@@ -59,7 +61,8 @@ struct MatchaArgs {
 struct PipePlan {
   int T, rows_per_item, n_slots, n_groups, smem_bytes, n_tiles, grid;  // all 0: the pipeline kernel did not run
   int head;        // columns [0, head) left to the direct-load kernel (a stream whose start is not 16-byte aligned)
-  int row_copies;  // 0: gradient rows travel as tensor-map boxes; 1: one bulk copy per row (rows not 16-byte aligned)
+  int row_copies;  // 0: gradient rows travel as tensor-map boxes; 1: one bulk copy per row (rows not 16-byte aligned);
+                   // 2: one bulk copy per row from a table of row pointers
   int x_stages;    // buffers of the step kernel's X stage (0 for the kernels that have none)
 };
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan);

@@ -35,6 +35,10 @@
 // memory, element by element.  The momentum and model rows are library-owned, 2 KB-pitched and keep
 // their box copies.  Same additions in the same order: identical bits.
 //
+// A third form (GM = kGPtrs) serves the streaming entry points in their "hold" mode: the finished
+// mini-batch gradients are separate 16-byte aligned vectors named by a table of row pointers; lane r
+// copies exactly its row's tile segment with one 1-D bulk copy and the consumers read it aligned.
+//
 // No CTA ever waits on another CTA.  Every mbarrier wait is bounded: after ~1 s of cycles a
 // waiting thread records an error code in global memory, all roles drain and the kernel returns
 // (the host reports it as an error status); nothing traps.
@@ -134,6 +138,10 @@ __device__ __forceinline__ void drain_and_exit_delay() {
 
 constexpr int kSmemBudget = 227 * 1024;
 constexpr int kMaxRowsPerItem = 8;
+// How the gradient rows of a ring item travel (template parameter GM):
+constexpr int kGBox = 0;   // 16-byte aligned strided stream: one tensor-map box of exactly r rows, issued by lane 0
+constexpr int kGRows = 1;  // strided stream whose rows are not 16-byte aligned: per row the aligned superset, read at a byte shift
+constexpr int kGPtrs = 2;  // a table of row pointers (16-byte aligned vectors): per row exactly its tile segment
 constexpr int kMaxGroups = 4;
 constexpr int kBoxInner = 256;  // a box is at most 256 elements wide: rows are described in units of T*es/256 bytes
 
@@ -207,14 +215,14 @@ __device__ __forceinline__ float4 sum_rows(float4 acc, const unsigned char *rowp
 
 // Bounds-checked build: everything the producer is about to use for one ring item - the slot, the
 // copy coordinates, and (per-row copies) the source span of this lane's row - is in range.
-template <int ES, bool GA>
+template <int ES, int GM>
 __device__ __forceinline__ bool dbg_item_ok(const PipeArgs &a, int T, int tile, int i, int m0, int rows, int lane,
                                             uint32_t sl, int NS, int off_slots, int slot_bytes, int total) {
   bool ok = dbg_check(sl < (uint32_t)NS && off_slots + (int)(sl + 1) * slot_bytes <= total, a.err, bounds::kRingSlot);
   ok = dbg_check(bounds::index_inside(tile, a.n_tiles) && bounds::index_inside(i, a.s.K) && m0 >= 0 && rows >= 0 &&
                      m0 + rows <= a.s.M && rows <= kMaxRowsPerItem,
                  a.err, bounds::kTileCoordinate) && ok;
-  if constexpr (!GA) {
+  if constexpr (GM == kGRows) {
     if (lane < rows) {
       const unsigned char *src = a.g_base + (int64_t)i * a.g_ld_k_bytes + (int64_t)(m0 + lane) * a.g_ld_m_bytes +
                                  (int64_t)tile * (T * ES);
@@ -223,23 +231,36 @@ __device__ __forceinline__ bool dbg_item_ok(const PipeArgs &a, int T, int tile, 
                                          a.s.ext.g_hi),
                      a.err, bounds::kGradientAddress) && ok;
     }
+  } else if constexpr (GM == kGPtrs) {
+    if (lane < rows) {  // the row is a vector of P elements of its own: the tile segment lies inside it, 16-byte aligned
+      const uintptr_t row = reinterpret_cast<uintptr_t>(a.s.row_ptrs[(int64_t)i * a.s.M + m0 + lane]);
+      ok = dbg_check(row != 0 && row % 16 == 0 && (a.s.row_col0 * ES) % 16 == 0 && (int64_t)(tile + 1) * T <= a.s.P, a.err,
+                     bounds::kGradientAddress) && ok;
+    }
   }
   return ok;
 }
 
-// Producer side of one ring item's gradient rows.  GA: lane 0 issues one box of exactly `rows` rows.
-// Otherwise lanes 0..rows-1 each fetch the aligned superset of one row's tile segment.
-template <int ES, bool GA>
+// Producer side of one ring item's gradient rows.  kGBox: lane 0 issues one box of exactly `rows` rows.
+// kGRows: lanes 0..rows-1 each fetch the aligned superset of one row's tile segment.  kGPtrs: lanes
+// 0..rows-1 each fetch exactly one row's tile segment from the vector the row-pointer table names.
+template <int ES, int GM>
 __device__ __forceinline__ void issue_rows(const PipeArgs &a, unsigned char *dst, int T, int tile, int i, int m0,
                                            int rows, int lane, uint64_t *bar) {
-  if constexpr (GA) {
+  if constexpr (GM == kGBox) {
     if (rows > 0) tma_load_3d(dst, &a.gmap[rows - 1], tile * kBoxInner, m0, i, bar);
-  } else {
+  } else if constexpr (GM == kGRows) {
     if (lane < rows) {
       const unsigned char *src = a.g_base + (int64_t)i * a.g_ld_k_bytes + (int64_t)(m0 + lane) * a.g_ld_m_bytes +
                                  (int64_t)tile * (T * ES);
       src -= reinterpret_cast<uintptr_t>(src) & 15;
       bulk_load_1d(dst + lane * (T * ES + 16), src, (uint32_t)(T * ES + 16), bar);
+    }
+  } else {
+    if (lane < rows) {
+      const unsigned char *src = reinterpret_cast<const unsigned char *>(a.s.row_ptrs[(int64_t)i * a.s.M + m0 + lane]) +
+                                 (a.s.row_col0 + (int64_t)tile * T) * ES;
+      bulk_load_1d(dst + lane * (T * ES), src, (uint32_t)(T * ES), bar);
     }
   }
 }
@@ -274,12 +295,14 @@ __host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, i
 
 // ES = bytes per gradient element (2: bf16, 4: fp32).
 // TT = tile width known at compile time (512, the usual shape: strides become immediates) or 0 (a.T).
-// GA = gradient rows are 16-byte aligned (box copies through tensor maps) or not (one bulk copy per row).
-template <int ES, bool MEAN, int TT, bool GA>
+// GM = how the gradient rows travel: kGBox, kGRows or kGPtrs (see above).
+template <int ES, bool MEAN, int TT, int GM>
 __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeline_kernel(const __grid_constant__ PipeArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
-  constexpr int kRowPad = GA ? 0 : 16;
+  constexpr bool GA = GM != kGRows;          // the consumers read the staged rows aligned
+  constexpr bool kWarpIssue = GM != kGBox;   // the whole producer warp issues (one copy per row)
+  constexpr int kRowPad = GM == kGRows ? 16 : 0;
   const StepArgs &s = a.s;
   const int K = s.K, T = TT ? TT : a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
   const int NSG = NS / NG;  // slots in each group's ring
@@ -340,7 +363,7 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
     // with the items of the learners i = g, g+NG, ... ; a slot is always filled for, and released
     // by, the same group, in order, which is what makes waiting on a phase parity unambiguous, and
     // a slow group never holds up the copies of another.
-    if (!GA || lane == 0) {
+    if (kWarpIssue || lane == 0) {
       const int g = warp;
       uint32_t slot = 0, phase = 0;
       for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x) {
@@ -350,12 +373,12 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
           do {
             const int rows = (n - m0 < R) ? (n - m0) : R;
             const uint32_t sl = (uint32_t)g * NSG + slot;
-            if constexpr (GA) ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2);
+            if constexpr (!kWarpIssue) ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2);
             else ok = __all_sync(0xffffffffu, mbar_wait(&empty[sl], phase ^ 1, a.err, 2));
             if (!ok) break;
             if constexpr (kDebug) {
-              ok = dbg_item_ok<ES, GA>(a, T, tile, i, m0, rows, lane, sl, NS, L.off_slots, L.slot_bytes, L.total);
-              if constexpr (!GA) ok = __all_sync(0xffffffffu, ok);
+              ok = dbg_item_ok<ES, GM>(a, T, tile, i, m0, rows, lane, sl, NS, L.off_slots, L.slot_bytes, L.total);
+              if constexpr (kWarpIssue) ok = __all_sync(0xffffffffu, ok);
               if (!ok) break;
             }
             unsigned char *dst = slots + (size_t)sl * L.slot_bytes;
@@ -363,8 +386,8 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
               mbar_expect_tx(&full[sl], (uint32_t)(rows * (T * ES + kRowPad) + (m0 == 0 ? T * 4 : 0)));
               if (m0 == 0) tma_load_2d(dst, &a.vmap, tile * kBoxInner, i, &full[sl]);
             }
-            if constexpr (!GA) __syncwarp();
-            issue_rows<ES, GA>(a, dst + T * 4, T, tile, i, m0, rows, lane, &full[sl]);
+            if constexpr (kWarpIssue) __syncwarp();
+            issue_rows<ES, GM>(a, dst + T * 4, T, tile, i, m0, rows, lane, &full[sl]);
             if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
             m0 += R;
           } while (m0 < n);
@@ -549,11 +572,13 @@ __host__ __device__ inline StreamLayout stream_layout(int T, int es, int R, int 
   return L;
 }
 
-template <int ES, int MODE, bool GA>
+template <int ES, int MODE, int GM>
 __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline_kernel(const __grid_constant__ PipeArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
-  constexpr int kRowPad = GA ? 0 : 16;
+  constexpr bool GA = GM != kGRows;
+  constexpr bool kWarpIssue = GM != kGBox;
+  constexpr int kRowPad = GM == kGRows ? 16 : 0;
   const StepArgs &s = a.s;
   const int K = s.K, T = a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
   const int NSG = NS / NG;
@@ -575,7 +600,7 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
   bool ok = true;
 
   if (warp < NG) {
-    if (!GA || lane == 0) {  // producer of group `warp`
+    if (kWarpIssue || lane == 0) {  // producer of group `warp`
       const int g = warp;
       uint32_t slot = 0, phase = 0;
       for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x) {
@@ -585,17 +610,17 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
           do {
             const int rows = (n - m0 < R) ? (n - m0) : R;
             const uint32_t sl = (uint32_t)g * NSG + slot;
-            if constexpr (GA) ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2);
+            if constexpr (!kWarpIssue) ok = mbar_wait(&empty[sl], phase ^ 1, a.err, 2);
             else ok = __all_sync(0xffffffffu, mbar_wait(&empty[sl], phase ^ 1, a.err, 2));
             if (!ok) break;
             if constexpr (kDebug) {
-              ok = dbg_item_ok<ES, GA>(a, T, tile, i, m0, rows, lane, sl, NS, L.off_slots, L.slot_bytes, L.total);
-              if constexpr (!GA) ok = __all_sync(0xffffffffu, ok);
+              ok = dbg_item_ok<ES, GM>(a, T, tile, i, m0, rows, lane, sl, NS, L.off_slots, L.slot_bytes, L.total);
+              if constexpr (kWarpIssue) ok = __all_sync(0xffffffffu, ok);
               if (!ok) break;
             }
             if (lane == 0) mbar_expect_tx(&full[sl], (uint32_t)(rows * (T * ES + kRowPad)));  // 0 rows: a plain arrival
-            if constexpr (!GA) __syncwarp();
-            issue_rows<ES, GA>(a, slots + (size_t)sl * L.slot_bytes, T, tile, i, m0, rows, lane, &full[sl]);
+            if constexpr (kWarpIssue) __syncwarp();
+            issue_rows<ES, GM>(a, slots + (size_t)sl * L.slot_bytes, T, tile, i, m0, rows, lane, &full[sl]);
             if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
             m0 += R;
           } while (m0 < n);
@@ -765,6 +790,12 @@ struct Coverage {
 };
 Coverage coverage(const StepArgs &a, int es, int T) {
   Coverage c;
+  if (a.row_ptrs) {  // held rows: 16-byte aligned vectors, exact copies, every full tile
+    c.rows_aligned = true;
+    c.head = 0;
+    c.n_tiles = a.P / T;
+    return c;
+  }
   c.rows_aligned = (uintptr_t)a.G % 16 == 0 && (a.ld_m * es) % 16 == 0 && (a.ld_k * es) % 16 == 0;
   if (c.rows_aligned) {
     c.head = 0;
@@ -792,7 +823,7 @@ void fill_row_args(PipeArgs *p, const StepArgs &a, int es) {
 // apply (then the direct-load kernel runs the whole range).
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   PipeTuning &t = tuning();
-  if ((uintptr_t)a.G % es != 0) return false;
+  if (!a.row_ptrs && (uintptr_t)a.G % es != 0) return false;
   if (!encode_fn()) return false;
   int Rmax = t.rows ? t.rows : 8;
   if (Rmax < 1) Rmax = 1;
@@ -863,7 +894,7 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   plan->smem_bytes = L.total;
   plan->n_tiles = (int)cov.n_tiles;
   plan->head = (int)cov.head;
-  plan->row_copies = rows_aligned ? 0 : 1;
+  plan->row_copies = a.row_ptrs ? 2 : rows_aligned ? 0 : 1;
   plan->x_stages = x_stages;
   const int64_t max_ctas = (int64_t)ctas * t.sm_count;
   plan->grid = (int)(plan->n_tiles < max_ctas ? plan->n_tiles : max_ctas);
@@ -874,7 +905,7 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
 // 2 slots per group.
 bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   PipeTuning &t = tuning();
-  if ((uintptr_t)a.G % es != 0) return false;
+  if (!a.row_ptrs && (uintptr_t)a.G % es != 0) return false;
   if (!encode_fn()) return false;
   const int T = 512;
   const Coverage cov = coverage(a, es, T);
@@ -898,7 +929,7 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   plan->smem_bytes = stream_layout(T, es, R, slots, row_pad).total;
   plan->n_tiles = (int)cov.n_tiles;
   plan->head = (int)cov.head;
-  plan->row_copies = cov.rows_aligned ? 0 : 1;
+  plan->row_copies = a.row_ptrs ? 2 : cov.rows_aligned ? 0 : 1;
   plan->x_stages = 0;
   const int64_t max_ctas = (int64_t)ctas * t.sm_count;
   plan->grid = (int)(plan->n_tiles < max_ctas ? plan->n_tiles : max_ctas);
@@ -938,13 +969,14 @@ cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, 
                                    cudaStream_t st) {
   PipeArgs p;
   fill_pipe_args(&p, a, plan, err_flag);
-  if (plan.row_copies) fill_row_args(&p, a, es);
-  else if (!encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;  // nothing launched: caller falls back
+  if (plan.row_copies == 1) fill_row_args(&p, a, es);
+  else if (plan.row_copies == 0 && !encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;  // nothing launched: caller falls back
   const int threads = plan.n_groups * (32 + plan.T / 4);
-#define NB_LAUNCH(ES, MODE)                                                                               \
-  do {                                                                                                    \
-    if (plan.row_copies) nb_stream_pipeline_kernel<ES, MODE, false><<<plan.grid, threads, plan.smem_bytes, st>>>(p); \
-    else nb_stream_pipeline_kernel<ES, MODE, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);       \
+#define NB_LAUNCH(ES, MODE)                                                                                                       \
+  do {                                                                                                                            \
+    if (plan.row_copies == 2) nb_stream_pipeline_kernel<ES, MODE, kGPtrs><<<plan.grid, threads, plan.smem_bytes, st>>>(p);        \
+    else if (plan.row_copies == 1) nb_stream_pipeline_kernel<ES, MODE, kGRows><<<plan.grid, threads, plan.smem_bytes, st>>>(p);   \
+    else nb_stream_pipeline_kernel<ES, MODE, kGBox><<<plan.grid, threads, plan.smem_bytes, st>>>(p);                              \
   } while (0)
   if (es == 2) {
     if (centralized) NB_LAUNCH(2, kModeCentralized);
@@ -967,13 +999,15 @@ cudaError_t configure_pipeline() {
 #define NB_CFG1(...)                                                                                                  \
   if ((e = cudaFuncSetAttribute(__VA_ARGS__, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget)) != cudaSuccess) \
     return e;
-#define NB_CFG(ES, MEAN)                                                                   \
-  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, true>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, true>) \
-  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, false>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, false>)
+#define NB_CFG(ES, MEAN)                                                                                         \
+  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGBox>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, kGBox>)     \
+  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGRows>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, kGRows>)   \
+  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGPtrs>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, kGPtrs>)
   NB_CFG(2, true) NB_CFG(2, false) NB_CFG(4, true) NB_CFG(4, false)
 #undef NB_CFG
-#define NB_CFG(ES, MODE) \
-  NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, true>) NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, false>)
+#define NB_CFG(ES, MODE)                                                                                  \
+  NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGBox>) NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGRows>) \
+  NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGPtrs>)
   NB_CFG(2, kModeAccumulate) NB_CFG(2, kModeCentralized) NB_CFG(4, kModeAccumulate) NB_CFG(4, kModeCentralized)
 #undef NB_CFG
 #undef NB_CFG1
@@ -994,13 +1028,14 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
     if (!encode_map(&p.xmap, a.X, ub, 2, dims, strides, xbox) || !encode_map(&p.vmap, a.V, ub, 2, dims, strides, vbox))
       return cudaErrorNotSupported;  // nothing launched: caller falls back to the direct-load kernel
   }
-  if (plan.row_copies) fill_row_args(&p, a, es);
-  else if (!encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;
+  if (plan.row_copies == 1) fill_row_args(&p, a, es);
+  else if (plan.row_copies == 0 && !encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;
   const int threads = 32 + plan.n_groups * (32 + plan.T / 4);  // X producer + per group: producer warp + consumers
 #define NB_LAUNCH2(ES, MEAN, TT)                                                                                   \
   do {                                                                                                             \
-    if (plan.row_copies) nb_step_pipeline_kernel<ES, MEAN, TT, false><<<plan.grid, threads, plan.smem_bytes, st>>>(p); \
-    else nb_step_pipeline_kernel<ES, MEAN, TT, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);              \
+    if (plan.row_copies == 2) nb_step_pipeline_kernel<ES, MEAN, TT, kGPtrs><<<plan.grid, threads, plan.smem_bytes, st>>>(p);      \
+    else if (plan.row_copies == 1) nb_step_pipeline_kernel<ES, MEAN, TT, kGRows><<<plan.grid, threads, plan.smem_bytes, st>>>(p); \
+    else nb_step_pipeline_kernel<ES, MEAN, TT, kGBox><<<plan.grid, threads, plan.smem_bytes, st>>>(p);                            \
   } while (0)
 #define NB_LAUNCH(ES, MEAN)                       \
   do {                                            \

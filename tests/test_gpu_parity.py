@@ -371,6 +371,85 @@ def test_host_buffer_entry_point(B):
     a.close(); b.close()
 
 
+@pytest.mark.parametrize("variant,order,K,P,dtype", [
+    ("dpsgd", 0, 16, 3 * 512 + 20, "bf16"), ("dpsgd", 1, 16, 2 * 512 + 7, "bf16"), ("allreduce", 0, 8, 5 * 512, "f32"),
+    ("allreduce", 1, 33, 512 + 100, "f32"), ("centralized", 0, 8, 4 * 512 + 9, "bf16"), ("dpsgd", 0, 64, 2 * 512 + 33, "bf16"),
+    ("dpsgd", 0, 5, 300, "f32"),
+])
+def test_streaming_hold_mode_reads_the_delivered_vectors_in_place(B, variant, order, K, P, dtype):
+    """NB_STREAMING_HOLD: deliveries are only recorded and nb_step runs the fused step on the vectors
+    where they lie (separate allocations, one per mini-batch gradient).  Same terminal-signal
+    behaviour as the accumulate mode (Alg. 1 inner loop), the same bits as that mode, oracle parity."""
+    import torch
+    M = 6
+    rng = np.random.default_rng(K * 1000 + P)
+    topo = B.make_topology("ring") if variant == "dpsgd" else None
+    hold, acc = B.NbContext(K, P, M, 0.05, 0.9, variant, topo), B.NbContext(K, P, M, 0.05, 0.9, variant, topo)
+    hold.set_option(B.NB_OPT_STREAMING, B.NB_STREAMING_HOLD)
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    for c in (hold, acc):
+        if variant != "centralized":
+            c.set_option(B.NB_OPT_ORDER, order)
+        c.set_params(torch.from_numpy(x0).cuda())
+    if variant == "centralized":
+        orc = None
+        x_ps, v_ps = x0.astype(np.float64), np.zeros(P)
+    else:
+        W = O.ring_W(K) if variant == "dpsgd" else None
+        orc = O.Oracle(K, P, M, 0.05, 0.9, "dpsgd" if variant == "dpsgd" else "allreduce", W=W,
+                       order="mix_then_update" if order == 0 else "update_then_mix")
+        orc.set_params(x0)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    for t in range(3):
+        n = rng.integers(0, M + 1, K)
+        n[int(rng.integers(0, K))] = M                               # someone finishes: the terminal signal is raised
+        # one separate device allocation per mini-batch gradient (what a learner would hand over)
+        vecs = [[(torch.from_numpy(rng.standard_normal(P).astype(np.float32)) * 0.01).to(tdt).cuda() for _ in range(M)]
+                for _ in range(K)]
+        for c in (hold, acc):
+            c.begin_iteration()
+        done_first = None
+        for m in range(M):                                           # round-robin arrival, as in a real iteration
+            for i in range(K):
+                if m < n[i]:
+                    ra, rb = hold.accumulate_minibatch(i, vecs[i][m]), acc.accumulate_minibatch(i, vecs[i][m])
+                    assert ra == rb
+        assert hold.get_finished()[0].tolist() == acc.get_finished()[0].tolist()
+        got_n = hold.get_finished()[0]
+        hold.step(); acc.step()
+        torch.cuda.synchronize()                                     # the vectors may be released only now
+        G = torch.stack([torch.stack(v) for v in vecs]).float().cpu().numpy()
+        if orc is not None:
+            orc.step(G, got_n.tolist())
+        else:
+            x_ps, v_ps = O.step_centralized(x_ps, v_ps, G, got_n.tolist(), 0.05, 0.9)
+    assert torch.equal(hold.get_params(), acc.get_params()) and torch.equal(hold.get_momentum(), acc.get_momentum())
+    if orc is not None:
+        H.assert_close(hold.get_params().numpy(), orc.X, H.TOL_SAME_INPUT)
+        H.assert_close(hold.get_momentum().numpy(), orc.V, H.TOL_SAME_INPUT)
+    else:
+        H.assert_close(hold.get_params().numpy(), x_ps, H.TOL_SAME_INPUT)
+    if P >= 1024:
+        assert hold.get_kernel_plan()["row_copies"] == 2 or variant == "centralized"
+    hold.check_guards()
+    # misuse: a vector that is not 16-byte aligned, a second dtype inside one iteration, a mode switch inside one
+    hold.begin_iteration()
+    flat = torch.zeros(P + 8, dtype=tdt, device="cuda")
+    with pytest.raises(B.NbError) as e:
+        hold.accumulate_minibatch(0, flat[1:P + 1])
+    assert e.value.code == B.NB_ERR_ARG
+    assert hold.accumulate_minibatch(0, flat[:P])
+    other = torch.zeros(P, dtype=torch.float32 if dtype == "bf16" else torch.bfloat16, device="cuda")
+    with pytest.raises(B.NbError) as e:
+        hold.accumulate_minibatch(0, other)
+    assert e.value.code == B.NB_ERR_ARG
+    with pytest.raises(B.NbError) as e:
+        hold.set_option(B.NB_OPT_STREAMING, B.NB_STREAMING_ACCUMULATE)
+    assert e.value.code == B.NB_ERR_STATE
+    hold.step()
+    hold.close(); acc.close()
+
+
 def test_error_reporting(B):
     import torch
     ctx = B.NbContext(4, 100, 4, 0.1, 0.9, "allreduce")
