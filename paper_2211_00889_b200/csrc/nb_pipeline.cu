@@ -846,8 +846,14 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
                                            {256, 1, 4, 2, 8}, {128, 1, 4, 2, 8}};
   static const Shape update_first_shapes[] = {{512, 1, 4, 3, 8}, {512, 2, 2, 2, 8}, {512, 1, 4, 2, 8}, {512, 1, 4, 1, 8},
                                               {512, 1, 4, 1, 4}, {256, 1, 4, 2, 8}, {128, 1, 4, 2, 8}};
+  // Few mini-batches per batch (items of a momentum row and at most 4 KB of gradient rows): one CTA
+  // per SM with four groups and three slots per group (cfg4 sizes at P = 138M: 0.99 of the measured
+  // copy bandwidth against 0.95 for two CTAs with two groups of two slots; equal within 1 % at 25-51M).
+  static const Shape small_item_shapes[] = {{512, 1, 4, 2, 8}, {512, 2, 2, 2, 8}, {512, 1, 4, 1, 8}, {512, 1, 4, 1, 4},
+                                            {256, 1, 4, 2, 8}, {128, 1, 4, 2, 8}};
   const bool mix_first = a.order == NB_ORDER_MIX_THEN_UPDATE;
-  const Shape *shapes = mix_first ? mix_first_shapes : update_first_shapes;
+  const bool small_items = mix_first && slot_bytes_of(512 * 4, 512, es, Rmax, row_pad) <= 6400;  // <= 4 bf16 / 2 fp32 rows
+  const Shape *shapes = small_items ? small_item_shapes : mix_first ? mix_first_shapes : update_first_shapes;
   const int n_shapes = mix_first ? 6 : 7;
   int T = 0, ctas = 0, groups = 0, slots = 0, x_stages = 0, R = Rmax;
   bool found = false;
@@ -877,14 +883,16 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   if (cov.n_tiles < 1) return false;
   if ((cov.n_tiles + 1) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
   // Ring depth.  With two X buffers in the Alg. 2 order, when one item holds a learner's whole
-  // contribution (R >= M) two slots per group keep the copies back to back and deeper rings measured
+  // contribution (R >= M) two slots per group (three for the small items of M <= 4) keep the copies
+  // back to back and deeper rings measured
   // 1-4 % slower (more copies in flight than the latency needs only spread the chip over more DRAM
   // rows at once); learners that need several items per tile use all the slots that fit.  Every slot
   // that fits is also used by the shapes whose consumers pause: the single X buffer of K > 32 (the ring
   // is what keeps memory busy while the next tile's models load: K = 40 / 48, 12 slots 1.03 of the
   // measured copy bandwidth, 8 slots 0.98) and the update-then-mix order (no slot is released while a
   // group averages: cfg3 sizes 12 slots 1.04, 8 slots 0.99).
-  if (!t.slots && mix_first && x_stages == 2 && R >= a.M && slots > 2 * groups) slots = 2 * groups;
+  const int per_group = (small_items && ctas == 1) ? 3 : 2;
+  if (!t.slots && mix_first && x_stages == 2 && R >= a.M && slots > per_group * groups) slots = per_group * groups;
   const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots, row_pad, x_stages);
   if (L.total > kSmemBudget) return false;
   plan->T = T;
