@@ -48,9 +48,10 @@ TRAFFIC_PER_ALGORITHMIC_BYTE = {
     "cfg3_dpsgd_ring_resnet50[P+1, rows not 16-byte aligned]": 0.988,
     "cfg3_dpsgd_ring_resnet50[update_then_mix]": 0.987,
     "cfg3_dpsgd_ring_resnet50[unfused]": 1.284,
+    "cfg3_dpsgd_ring_resnet50[streaming_hold]": 0.988,
     "cfg3_dpsgd_ring_resnet50[centralized]": 0.997,
     "cfg2_allreduce_resnet18": 0.990,
-    "cfg4_matcha_vgg16": 0.980,
+    "cfg4_matcha_vgg16": 0.981,
     "cfg5_scale_allreduce": 0.990,
     "cfg5_scale_ring": 0.990,
     "ring_K64_P12.8M": 0.987,

@@ -246,7 +246,7 @@ int nb_accumulate(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t
 /* Row pitch, in elements, at which a gradient stream of P columns of `dtype` streams fastest: the
  * smallest multiple of 2 KB that holds P elements.  Every 512-column tile segment of every row then
  * lies inside one 2 KB block of device memory (measured on B200, P = 138,000,000 bf16: dense rows,
- * whose segments straddle those blocks, run 2.7 % below rows at this pitch).  Pass it as ld_m (and
+ * whose segments straddle those blocks, run 1 to 3 % below rows at this pitch).  Pass it as ld_m (and
  * M * pitch, or more, as ld_k).  Purely advisory: any pitch >= P is accepted.  Returns 0 for P < 1
  * or an unknown dtype. */
 int64_t nb_recommended_pitch(int64_t P, int dtype);
