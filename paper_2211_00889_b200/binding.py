@@ -263,7 +263,8 @@ class NbContext:
 
     def close(self):
         if getattr(self, "_h", None):
-            lib.nb_destroy(self._h)
+            if lib is not None:          # (None while the interpreter is shutting down: the process frees the GPU itself)
+                lib.nb_destroy(self._h)
             self._h = None
 
     __del__ = close

@@ -909,8 +909,8 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   return true;
 }
 
-// Shape of the no-stage kernel: T = 512, R rows per item, as many CTAs per SM as keep at least
-// 2 slots per group.
+// Shape of the no-stage kernels: T = 512, R rows per item; two CTAs per SM with two groups each for
+// the masked accumulate, four CTAs of one group for the centralized step.
 bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   PipeTuning &t = tuning();
   if (!a.row_ptrs && (uintptr_t)a.G % es != 0) return false;
@@ -922,12 +922,21 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   const int row_pad = cov.rows_aligned ? 0 : 16;
   int R = es == 2 ? 8 : 4;
   if (R > a.M) R = a.M;
-  int groups = centralized ? 1 : 2;
+  int groups = centralized ? 1 : (t.groups ? t.groups : 2);
+  if (groups > kMaxGroups) groups = kMaxGroups;
   if (groups > a.K) groups = a.K;
-  const int ctas = centralized ? 4 : 2;
+  const int ctas = t.ctas_per_sm ? t.ctas_per_sm : centralized ? 4 : 2;
   const int budget = kSmemBudget / ctas - 1024;
   int slots = (budget - 512) / slot_bytes_of(0, T, es, R, row_pad);
   if (slots > 16) slots = 16;
+  if (!centralized) {
+    // Masked accumulate: about 32 KB of ring per group is the optimum (cfg3 sizes, 8 KB slots, slots per
+    // CTA -> fraction of the measured copy bandwidth: 4 -> 0.86, 6 -> 1.01, 8 -> 1.05, 12 -> 0.91).
+    int per_group = 32768 / slot_bytes_of(0, T, es, R, row_pad);
+    if (per_group < 2) per_group = 2;
+    if (slots > per_group * groups) slots = per_group * groups;
+  }
+  if (t.slots && t.slots < slots) slots = t.slots;
   slots -= slots % groups;
   if (slots < 2 * groups) return false;
   plan->T = T;
