@@ -853,7 +853,10 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
                                             {256, 1, 4, 2, 8}, {128, 1, 4, 2, 8}};
   const bool mix_first = a.order == NB_ORDER_MIX_THEN_UPDATE;
   const bool small_items = mix_first && slot_bytes_of(512 * 4, 512, es, Rmax, row_pad) <= 6400;  // <= 4 bf16 / 2 fp32 rows
-  const Shape *shapes = small_items ? small_item_shapes : mix_first ? mix_first_shapes : update_first_shapes;
+  // Rows named by a pointer table (the streaming entry points in hold mode) also do best on one CTA per SM
+  // with four groups (cfg3 sizes: 0.99 against 0.98 for two CTAs of two groups).
+  const bool one_cta_first = small_items || (mix_first && a.row_ptrs != nullptr);
+  const Shape *shapes = one_cta_first ? small_item_shapes : mix_first ? mix_first_shapes : update_first_shapes;
   const int n_shapes = mix_first ? 6 : 7;
   int T = 0, ctas = 0, groups = 0, slots = 0, x_stages = 0, R = Rmax;
   bool found = false;
@@ -910,7 +913,7 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
 }
 
 // Shape of the no-stage kernels: T = 512, R rows per item; two CTAs per SM with two groups each for
-// the masked accumulate, four CTAs of one group for the centralized step.
+// the masked accumulate, six CTAs of one group for the centralized step.
 bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   PipeTuning &t = tuning();
   if (!a.row_ptrs && (uintptr_t)a.G % es != 0) return false;
@@ -925,7 +928,10 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   int groups = centralized ? 1 : (t.groups ? t.groups : 2);
   if (groups > kMaxGroups) groups = kMaxGroups;
   if (groups > a.K) groups = a.K;
-  const int ctas = t.ctas_per_sm ? t.ctas_per_sm : centralized ? 4 : 2;
+  // centralized step, CTAs per SM -> fraction of the measured copy bandwidth (cfg3 sizes): 3 -> 0.89, 4 -> 1.02, 5 -> 1.045,
+  // 6 -> 1.05, 7 -> 0.77 (three slots each), 8 -> 0.83
+  // (fp32 gradients, cfg2 sizes: 4 -> 1.01, 5 -> 0.86, 6 -> 0.97; items of 2.5 KB, cfg4 sizes: 4 -> 0.69, 6 -> 0.81)
+  const int ctas = t.ctas_per_sm ? t.ctas_per_sm : centralized ? (es == 2 ? 6 : 4) : 2;
   const int budget = kSmemBudget / ctas - 1024;
   int slots = (budget - 512) / slot_bytes_of(0, T, es, R, row_pad);
   if (slots > 16) slots = 16;
