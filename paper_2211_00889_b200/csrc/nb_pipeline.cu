@@ -938,8 +938,10 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   if (!centralized) {
     // Masked accumulate: about 32 KB of ring per group is the optimum (cfg3 sizes, 8 KB slots, slots per
     // CTA -> fraction of the measured copy bandwidth: 4 -> 0.86, 6 -> 1.01, 8 -> 1.05, 12 -> 0.91).
+    // (4 KB slots, cfg4 sizes, slots per CTA: 8 -> 0.94, 12 -> 1.00, 14 -> 0.97, 16 -> 0.94: at most 6 per group)
     int per_group = 32768 / slot_bytes_of(0, T, es, R, row_pad);
     if (per_group < 2) per_group = 2;
+    if (per_group > 6) per_group = 6;
     if (slots > per_group * groups) slots = per_group * groups;
   }
   if (t.slots && t.slots < slots) slots = t.slots;
