@@ -350,9 +350,10 @@ int nb_debug_index_code(int64_t index, int64_t count);
  * everything; [1] tile width in columns; [2] consumer groups per CTA; [3] ring slots per CTA;
  * [4] gradient rows per ring item; [5] CTAs launched; [6] dynamic shared memory per CTA in bytes;
  * [7] tiles covered; [8] 0 if the gradient rows travelled as tensor-map boxes, 1 if as one bulk
- * copy per row (rows not 16-byte aligned); [9] columns before the first covered tile (they, and the
+ * copy per row (rows not 16-byte aligned), 2 if as one bulk copy per held vector (NB_STREAMING_HOLD);
+ * [9] columns before the first covered tile (they, and the
  * columns after [9] + [7]*[1], went to the direct-load kernel); [10] buffers of the old-model stage
- * (1-3); [11] reserved, 0. */
+ * (1-3; 0 for the centralized step, which has none); [11] columns a consumer thread owns (4 or 8). */
 int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan);
 
 /* ------------------------------------------------------------------------------------------------

@@ -396,7 +396,7 @@ class NbContext:
         a = np.zeros(12, dtype=np.int32)
         self._ck(lib.nb_get_kernel_plan(self._h, _i32p(a)))
         keys = ("pipeline", "tile", "groups", "slots", "rows_per_item", "grid", "smem_bytes", "tiles", "row_copies",
-                "head", "x_buffers", "reserved")
+                "head", "x_buffers", "columns_per_thread")
         return dict(zip(keys, (int(v) for v in a)))
 
     def get_stats(self):

@@ -223,7 +223,7 @@ int launch_update(nb_ctx *c, const nb::StepArgs &a, int src, cudaStream_t st) {
   int n_launched = 0;
   const bool pipeline = c->kernel == NB_KERNEL_AUTO;
   cudaError_t e;
-  if (c->variant == NB_CENTRALIZED) e = nb::launch_centralized(a, src, pipeline, c->d_err, &n_launched, st);
+  if (c->variant == NB_CENTRALIZED) e = nb::launch_centralized(a, src, pipeline, c->d_err, &n_launched, &c->last_plan, st);
   else e = nb::launch_step(a, src, pipeline, c->d_err, &n_launched, &c->last_plan, st);
   c->launches += n_launched;
   if (e != cudaSuccess) return cuda_fail(c, e, "launch_step");
@@ -801,7 +801,7 @@ int nb_get_kernel_plan(const nb_ctx *c, int32_t *plan) {
   plan[8] = p.row_copies;
   plan[9] = p.head;
   plan[10] = p.x_stages;
-  plan[11] = 0;
+  plan[11] = p.n_tiles > 0 ? 4 * p.quads_per_thread : 0;
   return NB_OK;
 }
 

@@ -539,13 +539,14 @@ cudaError_t launch_step(const StepArgs &a, int src, bool pipeline, int *err_flag
       });
 }
 
-cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, cudaStream_t st) {
+cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, PipePlan *used,
+                               cudaStream_t st) {
   const int es = src == kSrcBF16 ? 2 : 4;
   const StepArgs p = src == kSrcAcc ? acc_as_stream(a) : a;
   PipePlan plan;
   const bool planned = pipeline && plan_stream(p, es, true, &plan);
   return cover_columns(
-      a, p, es, planned ? &plan : nullptr, launches, nullptr,
+      a, p, es, planned ? &plan : nullptr, launches, used,
       [&](const StepArgs &r, const PipePlan &pl) { return launch_stream_pipeline(r, es, true, pl, err_flag, st); },
       [&](const StepArgs &r) {
         if (pipeline && r.P <= kTailMaxColumns) return launch_tail(r, src, kTailCentralized, st);

@@ -64,6 +64,7 @@ struct PipePlan {
   int row_copies;  // 0: gradient rows travel as tensor-map boxes; 1: one bulk copy per row (rows not 16-byte aligned);
                    // 2: one bulk copy per row from a table of row pointers
   int x_stages;    // buffers of the step kernel's X stage (0 for the kernels that have none)
+  int quads_per_thread = 1;  // groups of four columns per consumer thread (no-stage kernels: 1 or 2)
 };
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan);
 bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan);
@@ -89,7 +90,8 @@ cudaError_t launch_step(const StepArgs &a, int src, bool pipeline, int *err_flag
 cudaError_t launch_step_direct_only(const StepArgs &a, int src, cudaStream_t st);
 cudaError_t launch_add_minibatch(float *acc_row, const void *g, int src, bool aligned, int64_t P, bool first,
                                  const bounds::Extents &ext, int *err, cudaStream_t st);
-cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, cudaStream_t st);
+cudaError_t launch_centralized(const StepArgs &a, int src, bool pipeline, int *err_flag, int *launches, PipePlan *used,
+                               cudaStream_t st);
 cudaError_t launch_matcha_build(const MatchaArgs &a, cudaStream_t st);
 cudaError_t launch_mean(const float *X, int64_t ldx, int K, int64_t P, float *out, const bounds::Extents &ext, int *err,
                         cudaStream_t st);

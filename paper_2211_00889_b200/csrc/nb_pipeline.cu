@@ -558,6 +558,7 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
 // the direct-load kernel does.
 // -------------------------------------------------------------------------------------------------
 constexpr int kModeAccumulate = 0, kModeCentralized = 1;
+constexpr int kStreamTile = 512;  // the only tile width the no-stage kernels use
 
 struct StreamLayout {
   int32_t off_slots, slot_bytes, total;
@@ -572,7 +573,9 @@ __host__ __device__ inline StreamLayout stream_layout(int T, int es, int R, int 
   return L;
 }
 
-template <int ES, int MODE, int GM>
+// QPT: groups of four columns a consumer thread owns (T / QPT apart, so that a warp's accesses stay
+// contiguous); a group has T / (4 QPT) consumer threads.
+template <int ES, int MODE, int GM, int QPT>
 __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline_kernel(const __grid_constant__ PipeArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
@@ -580,18 +583,19 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
   constexpr bool kWarpIssue = GM != kGBox;
   constexpr int kRowPad = GM == kGRows ? 16 : 0;
   const StepArgs &s = a.s;
-  const int K = s.K, T = a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
+  constexpr int T = kStreamTile;  // strides and offsets become immediates
+  const int K = s.K, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
   const int NSG = NS / NG;
   const StreamLayout L = stream_layout(T, ES, R, NS, kRowPad);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);
   uint64_t *empty = full + NS;
   unsigned char *slots = smem_raw + L.off_slots;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int group_warps = T / 128;
+  const int group_threads = T / (4 * QPT);
   if (threadIdx.x == 0) {
     for (int q = 0; q < NS; ++q) {
       mbar_init(&full[q], 1);
-      mbar_init(&empty[q], group_warps);
+      mbar_init(&empty[q], group_threads / 32);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -629,27 +633,38 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
     }
   } else {
     const int ct = threadIdx.x - 32 * NG;
-    const int nq = T / 4;
-    const int grp = ct / nq, cq = ct - grp * nq;
+    const int grp = ct / group_threads, cq = ct - grp * group_threads;
     uint32_t slot = 0, phase = 0;
     for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x) {
-      const int64_t col0 = (int64_t)tile * T + (int64_t)cq * 4;
-      float4 x = make_float4(0.f, 0.f, 0.f, 0.f), v = x, gs = x;
+      const int64_t col0 = (int64_t)tile * T + (int64_t)cq * 4;  // this thread's q-th column group starts at col0 + q T / QPT
+      float4 x[QPT], v[QPT], gs[QPT];
+#pragma unroll
+      for (int q = 0; q < QPT; ++q) x[q] = v[q] = gs[q] = make_float4(0.f, 0.f, 0.f, 0.f);
       if constexpr (kDebug) {  // this thread's global footprint of the tile
-        const bool in = MODE == kModeAccumulate
-                            ? dbg_rows_inside(s.acc, ldx, K, col0, 4, 4, s.ext.acc_lo, s.ext.acc_hi)
-                            : dbg_rows_inside(s.X, ldx, 1, col0, 4, 4, s.ext.x_lo, s.ext.x_hi) &&
-                                  dbg_rows_inside(s.V, ldx, 1, col0, 4, 4, s.ext.v_lo, s.ext.v_hi);
+        bool in = true;
+#pragma unroll
+        for (int q = 0; q < QPT; ++q) {
+          const int64_t c = col0 + q * (T / QPT);
+          in = in && (MODE == kModeAccumulate
+                          ? dbg_rows_inside(s.acc, ldx, K, c, 4, 4, s.ext.acc_lo, s.ext.acc_hi)
+                          : dbg_rows_inside(s.X, ldx, 1, c, 4, 4, s.ext.x_lo, s.ext.x_hi) &&
+                                dbg_rows_inside(s.V, ldx, 1, c, 4, 4, s.ext.v_lo, s.ext.v_hi));
+        }
         ok = __all_sync(0xffffffffu, dbg_check(in, a.err, bounds::kStateAddress));
         if (!ok) break;
       }
       if constexpr (MODE == kModeCentralized) {  // requested early, used after the last learner
-        x = ld4(s.X + col0);
-        v = ld4(s.V + col0);
+#pragma unroll
+        for (int q = 0; q < QPT; ++q) {
+          x[q] = ld4(s.X + col0 + q * (T / QPT));
+          v[q] = ld4(s.V + col0 + q * (T / QPT));
+        }
       }
       for (int i = grp; ok && i < K; i += NG) {
         const int n = s.n[i];
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 acc[QPT];
+#pragma unroll
+        for (int q = 0; q < QPT; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         int m0 = 0;
         do {
           const int rows = (n - m0 < R) ? (n - m0) : R;
@@ -663,9 +678,17 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
           }
           const unsigned char *rowp = slots + (size_t)sl * L.slot_bytes + (size_t)cq * 4 * ES;
           const int s0 = GA ? 0 : (a.g_mis0 + i * a.g_mis_k + m0 * a.g_mis_m);
-          for (int r = 0; r < rows; ++r) {
-            const int shift = GA ? 0 : ((s0 + r * a.g_mis_m) & 15);
-            acc = add4(acc, ld_row4<SRC, GA>(rowp + (size_t)r * (T * ES + kRowPad) + shift));
+          if constexpr (MODE == kModeCentralized) {  // all loads of the item first (same additions, same order)
+#pragma unroll
+            for (int q = 0; q < QPT; ++q)
+              acc[q] = sum_rows<SRC, GA>(acc[q], rowp + q * (T / QPT) * ES, T * ES + kRowPad, rows, s0, a.g_mis_m);
+          } else {
+            for (int r = 0; r < rows; ++r) {
+              const int shift = GA ? 0 : ((s0 + r * a.g_mis_m) & 15);
+#pragma unroll
+              for (int q = 0; q < QPT; ++q)
+                acc[q] = add4(acc[q], ld_row4<SRC, GA>(rowp + q * (T / QPT) * ES + (size_t)r * (T * ES + kRowPad) + shift));
+            }
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&empty[sl]);
@@ -674,17 +697,22 @@ __global__ void __launch_bounds__(kMaxGroups * (32 + 128), 1) nb_stream_pipeline
         } while (m0 < n);
         if (!ok) break;
         if constexpr (MODE == kModeAccumulate) {
-          st4(s.acc + (int64_t)i * ldx + col0, acc);
+#pragma unroll
+          for (int q = 0; q < QPT; ++q) st4(s.acc + (int64_t)i * ldx + col0 + q * (T / QPT), acc[q]);
         } else {
           const float si = s.s[i];
-          gs = fma4(si, acc, gs);
+#pragma unroll
+          for (int q = 0; q < QPT; ++q) gs[q] = fma4(si, acc[q], gs[q]);
         }
       }
       if (!ok) break;
       if constexpr (MODE == kModeCentralized) {
-        const float4 vn = momentum(s.mom, v, s.inv_K, gs);
-        st4(s.V + col0, vn);
-        st4(s.X + col0, descend(x, s.lr, vn));
+#pragma unroll
+        for (int q = 0; q < QPT; ++q) {
+          const float4 vn = momentum(s.mom, v[q], s.inv_K, gs[q]);
+          st4(s.V + col0 + q * (T / QPT), vn);
+          st4(s.X + col0 + q * (T / QPT), descend(x[q], s.lr, vn));
+        }
       }
     }
   }
@@ -706,7 +734,7 @@ __global__ void nb_wait_selftest_kernel(int *err, int code, long long limit_cycl
 }
 
 struct PipeTuning {
-  int T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0, x_stages = 0;
+  int T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0, x_stages = 0, qpt = 0;
   int sm_count = 0;
 };
 
@@ -726,6 +754,7 @@ PipeTuning &tuning() {
     q.rows = geti("NB_PIPELINE_ROWS", 0);
     q.groups = geti("NB_PIPELINE_GROUPS", 0);
     q.x_stages = geti("NB_PIPELINE_XSTAGES", 0);
+    q.qpt = geti("NB_PIPELINE_QPT", 0);
 #endif
     return q;
   }();
@@ -913,12 +942,12 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
 }
 
 // Shape of the no-stage kernels: T = 512, R rows per item; two CTAs per SM with two groups each for
-// the masked accumulate, six CTAs of one group for the centralized step.
+// the masked accumulate, CTAs of one group for the centralized step.
 bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   PipeTuning &t = tuning();
   if (!a.row_ptrs && (uintptr_t)a.G % es != 0) return false;
   if (!encode_fn()) return false;
-  const int T = 512;
+  const int T = kStreamTile;
   const Coverage cov = coverage(a, es, T);
   if (cov.n_tiles < 1) return false;
   if ((cov.n_tiles + 1) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
@@ -928,10 +957,14 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   int groups = centralized ? 1 : (t.groups ? t.groups : 2);
   if (groups > kMaxGroups) groups = kMaxGroups;
   if (groups > a.K) groups = a.K;
-  // centralized step, CTAs per SM -> fraction of the measured copy bandwidth (cfg3 sizes): 3 -> 0.89, 4 -> 1.02, 5 -> 1.045,
-  // 6 -> 1.05, 7 -> 0.77 (three slots each), 8 -> 0.83
-  // (fp32 gradients, cfg2 sizes: 4 -> 1.01, 5 -> 0.86, 6 -> 0.97; items of 2.5 KB, cfg4 sizes: 4 -> 0.69, 6 -> 0.81)
-  const int ctas = t.ctas_per_sm ? t.ctas_per_sm : centralized ? (es == 2 ? 6 : 4) : 2;
+  // Centralized step (one group per CTA).  bf16 gradients: 8 CTAs per SM whose consumer threads own two groups of four
+  // columns each (96 threads, 80 registers: 8 CTAs is what the register file holds).  Fraction of the measured copy
+  // bandwidth, cfg3 sizes / items of 2.5 KB (M = 4, cfg4 sizes): 6 CTAs of 4-column threads 1.05 / 0.89, 8 CTAs of
+  // 8-column threads 1.055 / 0.97 (6 such CTAs 1.04 / 0.78: the step is bound by the number of consumer groups
+  // and the instructions they issue per item, not by bytes in flight; ring depth beyond 4 slots changes nothing).
+  // fp32 gradients (cfg2 sizes): 4 CTAs of 4-column threads 1.01, 5 -> 0.86, 6 -> 0.97; 8-column threads 4 -> 1.02, 8 -> 0.93.
+  const int qpt = t.qpt ? (t.qpt == 2 ? 2 : 1) : (centralized && es == 2 ? 2 : 1);
+  const int ctas = t.ctas_per_sm ? t.ctas_per_sm : centralized ? (es == 2 ? 8 : 4) : 2;
   const int budget = kSmemBudget / ctas - 1024;
   int slots = (budget - 512) / slot_bytes_of(0, T, es, R, row_pad);
   if (slots > 16) slots = 16;
@@ -956,6 +989,7 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   plan->head = (int)cov.head;
   plan->row_copies = a.row_ptrs ? 2 : cov.rows_aligned ? 0 : 1;
   plan->x_stages = 0;
+  plan->quads_per_thread = qpt;
   const int64_t max_ctas = (int64_t)ctas * t.sm_count;
   plan->grid = (int)(plan->n_tiles < max_ctas ? plan->n_tiles : max_ctas);
   return true;
@@ -996,12 +1030,18 @@ cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, 
   fill_pipe_args(&p, a, plan, err_flag);
   if (plan.row_copies == 1) fill_row_args(&p, a, es);
   else if (plan.row_copies == 0 && !encode_gmaps(&p, a, es, plan)) return cudaErrorNotSupported;  // nothing launched: caller falls back
-  const int threads = plan.n_groups * (32 + plan.T / 4);
-#define NB_LAUNCH(ES, MODE)                                                                                                       \
-  do {                                                                                                                            \
-    if (plan.row_copies == 2) nb_stream_pipeline_kernel<ES, MODE, kGPtrs><<<plan.grid, threads, plan.smem_bytes, st>>>(p);        \
-    else if (plan.row_copies == 1) nb_stream_pipeline_kernel<ES, MODE, kGRows><<<plan.grid, threads, plan.smem_bytes, st>>>(p);   \
-    else nb_stream_pipeline_kernel<ES, MODE, kGBox><<<plan.grid, threads, plan.smem_bytes, st>>>(p);                              \
+  const int qpt = plan.quads_per_thread;
+  const int threads = plan.n_groups * (32 + plan.T / (4 * qpt));
+#define NB_LAUNCH1(ES, MODE, QPT)                                                                                                      \
+  do {                                                                                                                                 \
+    if (plan.row_copies == 2) nb_stream_pipeline_kernel<ES, MODE, kGPtrs, QPT><<<plan.grid, threads, plan.smem_bytes, st>>>(p);        \
+    else if (plan.row_copies == 1) nb_stream_pipeline_kernel<ES, MODE, kGRows, QPT><<<plan.grid, threads, plan.smem_bytes, st>>>(p);   \
+    else nb_stream_pipeline_kernel<ES, MODE, kGBox, QPT><<<plan.grid, threads, plan.smem_bytes, st>>>(p);                              \
+  } while (0)
+#define NB_LAUNCH(ES, MODE)                  \
+  do {                                       \
+    if (qpt == 2) NB_LAUNCH1(ES, MODE, 2);   \
+    else NB_LAUNCH1(ES, MODE, 1);            \
   } while (0)
   if (es == 2) {
     if (centralized) NB_LAUNCH(2, kModeCentralized);
@@ -1010,6 +1050,7 @@ cudaError_t launch_stream_pipeline(const StepArgs &a, int es, bool centralized, 
     if (centralized) NB_LAUNCH(4, kModeCentralized);
     else NB_LAUNCH(4, kModeAccumulate);
   }
+#undef NB_LAUNCH1
 #undef NB_LAUNCH
   return cudaGetLastError();
 }
@@ -1030,9 +1071,10 @@ cudaError_t configure_pipeline() {
   NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGPtrs>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, kGPtrs>)
   NB_CFG(2, true) NB_CFG(2, false) NB_CFG(4, true) NB_CFG(4, false)
 #undef NB_CFG
-#define NB_CFG(ES, MODE)                                                                                  \
-  NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGBox>) NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGRows>) \
-  NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGPtrs>)
+#define NB_CFG(ES, MODE)                                                                                            \
+  NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGBox, 1>) NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGRows, 1>)     \
+  NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGPtrs, 1>) NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGBox, 2>)     \
+  NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGRows, 2>) NB_CFG1(nb_stream_pipeline_kernel<ES, MODE, kGPtrs, 2>)
   NB_CFG(2, kModeAccumulate) NB_CFG(2, kModeCentralized) NB_CFG(4, kModeAccumulate) NB_CFG(4, kModeCentralized)
 #undef NB_CFG
 #undef NB_CFG1

@@ -71,6 +71,72 @@ def test_mid_size_every_column():
     ctx.close()
 
 
+@pytest.mark.parametrize("dtype,tiles", [("bf16", 3600), ("f32", 1800)])
+def test_mid_size_every_column_centralized(dtype, tiles):
+    """Alg. 3 on enough tiles that every CTA of the persistent no-stage kernel takes three or more
+    (ring phase wrap, the tile loop), every column compared with the oracle; and the same sizes through
+    nb_accumulate + nb_step (the masked-accumulate kernel in its persistent regime)."""
+    import torch
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    K, M, P = 8, 8, tiles * 512 + 24
+    rng = np.random.default_rng(tiles)
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    fused = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
+    unfused = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
+    for c in (fused, unfused):
+        c.set_params(torch.from_numpy(x0).cuda())
+    x, v = x0.astype(np.float64), np.zeros(P)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(tiles)
+    for t in range(3):
+        G = (torch.randn((K, M, P), generator=gen, device="cuda", dtype=torch.float32) * 0.01).to(tdt)
+        n = rng.integers(0, M + 1, K)
+        fused.step_fused(G, n)
+        plan = fused.get_kernel_plan()
+        unfused.accumulate(G, n)
+        unfused.step()
+        x, v = O.step_centralized(x, v, G.float().cpu().numpy(), n.tolist(), 0.1, 0.9)
+        del G
+    assert plan["pipeline"] == 1 and plan["tiles"] == tiles and plan["tiles"] >= 3 * plan["grid"]
+    H.assert_close(fused.get_params().numpy(), x, H.TOL_SAME_INPUT, "x")
+    H.assert_close(fused.get_momentum().numpy(), v, H.TOL_SAME_INPUT, "v")
+    assert torch.equal(fused.get_params(), unfused.get_params())
+    assert torch.equal(fused.get_momentum(), unfused.get_momentum())
+    for c in (fused, unfused):
+        c.check_guards()
+        c.close()
+
+
+def test_mid_size_every_column_update_then_mix():
+    """Eq. 4-6's order on 1200 tiles: the deferred averaging pass over three X buffers, every column."""
+    import torch
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 1200 * 512 + 24, steps=3)
+    ctx = B.context_for(w)
+    ctx.set_option(B.NB_OPT_ORDER, B.NB_ORDER_UPDATE_THEN_MIX)
+    orc = H.oracle_for(w, w.P, order="update_then_mix")
+    x0 = WL.init_params(w)
+    ctx.set_params(torch.from_numpy(x0).cuda())
+    orc.set_params(x0)
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        payload, values = WL.gradients_np(w, t)
+        ctx.step_fused(H.to_device(payload), n)
+        orc.step(values, n.tolist())
+        del payload, values
+    plan = ctx.get_kernel_plan()
+    assert plan["pipeline"] == 1 and plan["x_buffers"] == 3 and plan["tiles"] >= 3 * plan["grid"]
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT, "X")
+    H.assert_close(ctx.get_momentum().numpy(), orc.V, H.TOL_SAME_INPUT, "V")
+    ctx.check_guards()
+    ctx.close()
+
+
 def test_more_than_two_to_the_31_columns():
     """Column indices beyond 32 bits: one learner pair, 2^31 + 1544 columns (the last window the
     oracle checks lies entirely above 2^31)."""
