@@ -958,13 +958,20 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   if (groups > kMaxGroups) groups = kMaxGroups;
   if (groups > a.K) groups = a.K;
   // Centralized step (one group per CTA).  bf16 gradients: 8 CTAs per SM whose consumer threads own two groups of four
-  // columns each (96 threads, 80 registers: 8 CTAs is what the register file holds).  Fraction of the measured copy
+  // columns each (96 threads of 72 registers: nine such CTAs are what the register file holds).  Fraction of the measured copy
   // bandwidth, cfg3 sizes / items of 2.5 KB (M = 4, cfg4 sizes): 6 CTAs of 4-column threads 1.05 / 0.89, 8 CTAs of
   // 8-column threads 1.055 / 0.97 (6 such CTAs 1.04 / 0.78: the step is bound by the number of consumer groups
   // and the instructions they issue per item, not by bytes in flight; ring depth beyond 4 slots changes nothing).
   // fp32 gradients (cfg2 sizes): 4 CTAs of 4-column threads 1.01, 5 -> 0.86, 6 -> 0.97; 8-column threads 4 -> 1.02, 8 -> 0.93.
   const int qpt = t.qpt ? (t.qpt == 2 ? 2 : 1) : (centralized && es == 2 ? 2 : 1);
-  const int ctas = t.ctas_per_sm ? t.ctas_per_sm : centralized ? (es == 2 ? 8 : 4) : 2;
+  // Items of at most 5 KB (M <= 5) leave room for a ninth CTA (4-5 slots each): cfg4 sizes 0.97 -> 1.00, M = 1 / 2 0.55 ->
+  // 0.59 / 0.61, M = 5 1.00 -> 1.02, against 1.055 -> 1.045 for 8 KB items, which stay at eight.
+  // Masked accumulate: two CTAs of two groups (cfg3 sizes 1.05, M = 4 0.98-1.00); three when an item is at most 2 KB
+  // of bf16 rows (M = 1, 2: 0.79-0.80 -> 0.92-0.93).
+  const int item_bytes = slot_bytes_of(0, T, es, R, row_pad);
+  const int ctas = t.ctas_per_sm ? t.ctas_per_sm
+                   : centralized ? (es == 2 ? (item_bytes <= 5120 + 128 ? 9 : 8) : 4)
+                                 : (es == 2 && item_bytes <= 2048 + 128 ? 3 : 2);
   const int budget = kSmemBudget / ctas - 1024;
   int slots = (budget - 512) / slot_bytes_of(0, T, es, R, row_pad);
   if (slots > 16) slots = 16;
