@@ -8,7 +8,7 @@ Flavours (separate files, so that the shipped library is never replaced by one o
                    range-checked on the device; a failed check skips the access and records a code
                    in the context's device error word (reported as NB_ERR_CUDA by nb_check_guards)
   libnb_tuning.so  -DNB_TUNING: the pipeline planner reads shape overrides from the environment
-                   (NB_PIPELINE_TILE, _SLOTS, _CTAS_PER_SM, _ROWS, _GROUPS) for sweeps
+                   (NB_PIPELINE_TILE, _SLOTS, _CTAS_PER_SM, _ROWS, _GROUPS, _XSTAGES, _QPT) for sweeps
 The binding loads libnb.so unless the environment variable NB_LIB_PATH names another file.
 """
 import os

@@ -29,7 +29,7 @@
 //
 // Gradient rows whose byte addresses are not multiples of 16 (odd row lengths, a stream that starts
 // at an odd element) cannot be described by a tensor map.  They take the same path with one change
-// (template parameter GA = false): the producer WARP issues one plain 1-D bulk copy per finished row,
+// (template parameter GM = kGRows): the producer WARP issues one plain 1-D bulk copy per finished row,
 // lane r for row m0 + r, that fetches the 16-byte aligned superset of the row's tile segment (start
 // rounded down, T*ES + 16 bytes), and the consumers read each row at its own byte shift from shared
 // memory, element by element.  The momentum and model rows are library-owned, 2 KB-pitched and keep
