@@ -75,7 +75,8 @@ def test_mid_size_every_column():
 def test_mid_size_every_column_centralized(dtype, tiles):
     """Alg. 3 on enough tiles that every CTA of the persistent no-stage kernel takes three or more
     (ring phase wrap, the tile loop), every column compared with the oracle; and the same sizes through
-    nb_accumulate + nb_step (the masked-accumulate kernel in its persistent regime)."""
+    nb_accumulate + nb_step (the masked-accumulate kernel in its persistent regime), and from a stream
+    whose rows are not 16-byte aligned (one bulk copy per row), bit for bit."""
     import torch
     from paper_2211_00889_b200.build import build_library
     build_library()
@@ -85,7 +86,8 @@ def test_mid_size_every_column_centralized(dtype, tiles):
     x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
     fused = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
     unfused = B.NbContext(K, P, M, 0.1, 0.9, "centralized")
-    for c in (fused, unfused):
+    shifted = B.NbContext(K, P, M, 0.1, 0.9, "centralized")   # the same values one element off 16-byte alignment
+    for c in (fused, unfused, shifted):
         c.set_params(torch.from_numpy(x0).cuda())
     x, v = x0.astype(np.float64), np.zeros(P)
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
@@ -98,14 +100,25 @@ def test_mid_size_every_column_centralized(dtype, tiles):
         plan = fused.get_kernel_plan()
         unfused.accumulate(G, n)
         unfused.step()
+        flat = torch.empty(G.numel() + 1, dtype=G.dtype, device=G.device)
+        Gs = flat[1:].view_as(G)
+        Gs.copy_(G)
+        if t % 2:
+            shifted.step_fused(Gs, n)
+            assert shifted.get_kernel_plan()["row_copies"] == 1
+        else:
+            shifted.accumulate(Gs, n)
+            shifted.step()
+        del Gs, flat
         x, v = O.step_centralized(x, v, G.float().cpu().numpy(), n.tolist(), 0.1, 0.9)
         del G
     assert plan["pipeline"] == 1 and plan["tiles"] == tiles and plan["tiles"] >= 3 * plan["grid"]
     H.assert_close(fused.get_params().numpy(), x, H.TOL_SAME_INPUT, "x")
     H.assert_close(fused.get_momentum().numpy(), v, H.TOL_SAME_INPUT, "v")
-    assert torch.equal(fused.get_params(), unfused.get_params())
-    assert torch.equal(fused.get_momentum(), unfused.get_momentum())
-    for c in (fused, unfused):
+    for c in (unfused, shifted):
+        assert torch.equal(fused.get_params(), c.get_params())
+        assert torch.equal(fused.get_momentum(), c.get_momentum())
+    for c in (fused, unfused, shifted):
         c.check_guards()
         c.close()
 
