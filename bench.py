@@ -468,7 +468,33 @@ def other_workloads(args, B, WL, dev, base_runner, peak, local, log):
     run(w3.name + "[streaming_hold]", w3, entry="streaming_hold", bufs=shared,
         note="the same deliveries only recorded (NB_STREAMING_HOLD): nb_step runs the fused step on the delivered "
              "vectors where they lie, one bulk copy per row from a table of row pointers")
+    out.append(mean_model_entry(base_runner, peak, steps, local))
     return out, shared
+
+
+def mean_model_entry(runner, peak, steps, local):
+    """S7, the output step: nb_get_mean_params into a device buffer (K model rows read, one written)."""
+    torch, w, ctx = runner.torch, runner.w, runner.ctx
+    for _ in range(3):
+        ctx.get_mean_params(device=runner.dev)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record()
+    for _ in range(steps):
+        ctx.get_mean_params(device=runner.dev)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / steps
+    alg = 4.0 * w.P * (w.K + 1)
+    gbs = alg / (ms * 1e-3) / 1e9
+    return {"name": w.name + "[mean model]", "entry": "nb_get_mean_params", "steps": steps, "ms_per_step": ms,
+            "algorithmic_bytes_per_step": alg, "achieved_hbm_gbs": gbs, "frac": gbs / peak, "entry_moved_gbs": gbs,
+            "entry_moved_frac": gbs / peak, "traffic": None, "gpu_launches_per_step": 1.0, "kernel_plan": None,
+            "clocks": clocks,
+            "note": "Alg. 1 / Alg. 2 output: mean of the K learners' models, 4*P*(K+1) bytes"}
 
 
 def run_ours(args, w):
