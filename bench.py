@@ -589,9 +589,26 @@ def run_ours(args, w):
         wall = time.perf_counter() - t0
         dev_ms = a0.elapsed_time(a1)
         per = sharding.max_over_ranks(max(dev_ms, wall * 1e3), dev) / args.e2e_steps
+        # the bus roof beside it: one plain pinned host-to-device copy of 1 GiB, timed the same way
+        n_el = min(host.numel(), (1 << 30) // es)
+        dst = torch.empty(n_el, dtype=host.dtype, device=dev)
+        src = host.view(-1)[:n_el]
+        dst.copy_(src, non_blocking=True)
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b0.record()
+        for _ in range(3):
+            dst.copy_(src, non_blocking=True)
+        b1.record()
+        torch.cuda.synchronize()
+        pcie = 3 * n_el * es / (b0.elapsed_time(b1) * 1e-3) / 1e9
+        del dst, src
+        h2d_step = h2d // args.e2e_steps
         e2e = {"value": w.K * w.P * world / (per * 1e-3), "unit": UNIT, "ms_per_step": per,
-               "steps": args.e2e_steps, "h2d_bytes_per_step": h2d // args.e2e_steps,
+               "steps": args.e2e_steps, "h2d_bytes_per_step": h2d_step,
                "d2h_bytes_per_step": w.P * 4,
+               "h2d_gbs": h2d_step / (per * 1e-3) / 1e9, "plain_pinned_h2d_copy_gbs": pcie,
+               "bound": "host-to-device bus: only the finished rows cross it, overlapped with the kernels and the "
+                        "device-to-host copy of the mean model",
                "api": "nb_step_fused_host (pinned host gradients in, mean model out)"}
         del host, mean_out
         log("e2e done")
