@@ -885,8 +885,32 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   // Rows named by a pointer table (the streaming entry points in hold mode) also do best on one CTA per SM
   // with four groups (cfg3 sizes: 0.99 against 0.98 for two CTAs of two groups).
   const bool one_cta_first = small_items || (mix_first && a.row_ptrs != nullptr);
-  const Shape *shapes = one_cta_first ? small_item_shapes : mix_first ? mix_first_shapes : update_first_shapes;
-  const int n_shapes = mix_first ? 6 : 7;
+  const Shape *table = one_cta_first ? small_item_shapes : mix_first ? mix_first_shapes : update_first_shapes;
+  // Few learners: a tile carries few bytes (T (16 K + e_g sum n_i)), so what limits the step is how many tiles an SM
+  // has in flight, and the groups of one CTA share a single tile.  Four CTAs per SM of ONE consumer group each (the
+  // group takes all K learners of its tile) then do best.  Fraction of the measured copy bandwidth, ring, bf16, M = 1 /
+  // 4 / 8: K = 1 0.25 / 0.31 / 0.71 -> 0.71 / 0.88 / 0.97, K = 2 0.45 / 0.53 / 0.98 -> 0.85 / 0.94 / 1.02, K = 3 0.62 / 0.71 /
+  // 0.96 -> 0.88 / 0.96 / 1.03 (M <= 8: with two items per learner the tables' shapes stay ahead, K = 2, M = 16 0.99 against
+  // 0.94); with small items also K = 4..7 (K = 4 0.74 / 0.82 -> 0.90 / 0.97, K = 6 0.74 / 0.83 -> 0.91 /
+  // 0.98; their 8-row items stay at 1.03 on two CTAs of two groups, K = 8 at 0.92-1.04 on the tables above).
+  // Update-then-mix, K <= 8 (before: K = 2 0.37-0.55, K = 4 0.64-0.88, K = 6 0.64-0.86): four such CTAs, with three X
+  // buffers for K <= 2 and small items (K = 2 0.74-0.94, K = 4 0.84-1.00); K = 6, 7 with 8-row items two CTAs of two
+  // groups (0.86 -> 1.02); K = 8 with 8-row items keeps the table (1.02).
+  const bool small_slot = slot_bytes_of(512 * 4, 512, es, Rmax, row_pad) <= 6400;
+  Shape first = {0, 0, 0, 0, 0};
+  if (!a.row_ptrs) {
+    if (mix_first) {
+      if (a.K == 1 || (a.K <= 3 && Rmax >= a.M) || (a.K <= 7 && small_slot)) first = {512, 4, 1, 2, 8};
+    } else if (a.K <= 8) {
+      if (small_slot) first = {512, 4, 1, a.K <= 2 ? 3 : 2, 8};
+      else if (a.K <= 5) first = {512, 4, 1, 2, 8};
+      else if (a.K <= 7) first = {512, 2, 2, 2, 8};
+    }
+  }
+  Shape shapes[8];
+  int n_shapes = 0;
+  if (first.T) shapes[n_shapes++] = first;
+  for (int q = 0; q < (mix_first ? 6 : 7); ++q) shapes[n_shapes++] = table[q];
   int T = 0, ctas = 0, groups = 0, slots = 0, x_stages = 0, R = Rmax;
   bool found = false;
   for (int q = 0; q < n_shapes; ++q) {
