@@ -911,30 +911,42 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   int n_shapes = 0;
   if (first.T) shapes[n_shapes++] = first;
   for (int q = 0; q < (mix_first ? 6 : 7); ++q) shapes[n_shapes++] = table[q];
-  int T = 0, ctas = 0, groups = 0, slots = 0, x_stages = 0, R = Rmax;
-  bool found = false;
-  for (int q = 0; q < n_shapes; ++q) {
+  // The update-then-mix order releases no slot while a group averages, so its ring is what keeps memory busy: a shape is
+  // taken there only if the rings of an SM hold at least 56 KB (K = 32, M = 1: three X buffers leave 8 slots of 3 KB,
+  // 0.77; two leave 32, 0.96.  K = 40, M = 4: two buffers with 8 slots of 6 KB 0.81, one buffer with 24 0.90; K = 40,
+  // M = 1: two buffers with 20 slots of 3 KB 1.00); if no
+  // shape offers that, the first one that fits at all.
+  struct Chosen { int T, ctas, groups, slots, x_stages, R; };
+  Chosen c = {0, 0, 0, 0, 0, 0}, fallback = {0, 0, 0, 0, 0, 0};
+  for (int q = 0; q < n_shapes && !c.T; ++q) {
     const Shape &sh = shapes[q];
-    R = sh.rows < Rmax ? sh.rows : Rmax;
-    T = t.T ? t.T : sh.T;
-    ctas = t.ctas_per_sm ? t.ctas_per_sm : sh.ctas;
-    groups = t.groups ? t.groups : sh.groups;
-    x_stages = t.x_stages ? t.x_stages : sh.x_stages;
-    if (T != 128 && T != 256 && T != 512) return false;
-    if (x_stages < 1 || x_stages > kMaxXStages) return false;
-    if (groups > kMaxGroups) groups = kMaxGroups;
-    if (groups > a.K) groups = a.K;
-    while (groups > 1 && groups * (T / 4) > 512) --groups;
-    if (groups < 1 || ctas < 1) return false;
-    const PipeLayout L0 = pipe_layout(a.K, T, es, R, 0, a.mix_slots, row_pad, x_stages);
-    const int budget = kSmemBudget / ctas - 1024;
-    slots = (budget - L0.total - 256) / slot_bytes_of(T * 4, T, es, R, row_pad);
-    if (t.slots && t.slots < slots) slots = t.slots;
-    if (slots > 32) slots = 32;
-    slots -= slots % groups;  // every group's ring has the same number of slots
-    if (slots >= 2 * groups) { found = true; break; }
+    Chosen k;
+    k.R = sh.rows < Rmax ? sh.rows : Rmax;
+    k.T = t.T ? t.T : sh.T;
+    k.ctas = t.ctas_per_sm ? t.ctas_per_sm : sh.ctas;
+    k.groups = t.groups ? t.groups : sh.groups;
+    k.x_stages = t.x_stages ? t.x_stages : sh.x_stages;
+    if (k.T != 128 && k.T != 256 && k.T != 512) return false;
+    if (k.x_stages < 1 || k.x_stages > kMaxXStages) return false;
+    if (k.groups > kMaxGroups) k.groups = kMaxGroups;
+    if (k.groups > a.K) k.groups = a.K;
+    while (k.groups > 1 && k.groups * (k.T / 4) > 512) --k.groups;
+    if (k.groups < 1 || k.ctas < 1) return false;
+    const PipeLayout L0 = pipe_layout(a.K, k.T, es, k.R, 0, a.mix_slots, row_pad, k.x_stages);
+    const int budget = kSmemBudget / k.ctas - 1024;
+    const int slot_bytes = slot_bytes_of(k.T * 4, k.T, es, k.R, row_pad);
+    k.slots = (budget - L0.total - 256) / slot_bytes;
+    if (t.slots && t.slots < k.slots) k.slots = t.slots;
+    if (k.slots > 32) k.slots = 32;
+    k.slots -= k.slots % k.groups;  // every group's ring has the same number of slots
+    if (k.slots < 2 * k.groups) continue;
+    if (!fallback.T) fallback = k;
+    if (mix_first || t.slots || (int64_t)k.ctas * k.slots * slot_bytes >= 56 * 1024) c = k;
   }
-  if (!found) return false;
+  if (!c.T) c = fallback;
+  if (!c.T) return false;
+  const int T = c.T, ctas = c.ctas, groups = c.groups, x_stages = c.x_stages, R = c.R;
+  int slots = c.slots;
   const Coverage cov = coverage(a, es, T);
   if (cov.n_tiles < 1) return false;
   if ((cov.n_tiles + 1) * (int64_t)kBoxInner >= (1ll << 31)) return false;  // tile coordinates are 32-bit
