@@ -941,7 +941,11 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
     k.slots -= k.slots % k.groups;  // every group's ring has the same number of slots
     if (k.slots < 2 * k.groups) continue;
     if (!fallback.T) fallback = k;
-    if (mix_first || t.slots || (int64_t)k.ctas * k.slots * slot_bytes >= 56 * 1024) c = k;
+    // Alg. 2 order, learners that need several items per tile (M > R): two CTAs per SM are taken only with four slots
+    // per group (K = 16, M = 16, bf16: two slots per group 0.99, one CTA of four groups with every slot that fits 1.03).
+    const bool deep_enough = mix_first ? (k.ctas != 2 || k.R >= a.M || k.slots >= 4 * k.groups)
+                                       : (int64_t)k.ctas * k.slots * slot_bytes >= 56 * 1024;
+    if (deep_enough || t.slots) c = k;
   }
   if (!c.T) c = fallback;
   if (!c.T) return false;
