@@ -83,6 +83,8 @@ def parse_args():
     ap.add_argument("--no-sustained", action="store_true", help="skip the >= 2 s repetition of the headline step")
     ap.add_argument("--workload-steps", type=int, default=20, help="timed steps of every `workloads` entry")
     ap.add_argument("--sustained-seconds", type=float, default=2.5)
+    ap.add_argument("--coverage-map", action="store_true",
+                    help="instead of the benchmark: the fused step over a grid of K, M, dtype, variant and order")
     ap.add_argument("--cpu-sample-cols", type=int, default=4_000_000)
     ap.add_argument("--cpu-sample-steps", type=int, default=8)
     a = ap.parse_args()
@@ -701,9 +703,49 @@ def larger_workloads(args, B, WL, dev, w_head, peak, local, log):
     return out
 
 
+def coverage_map(args):
+    """`--coverage-map`: the fused step over a grid of K, M, gradient dtype, variant and order (10 timed
+    steps each, sizes of 5-8 GB), as fractions of the measured copy bandwidth; one JSON line.  Shows
+    where the planner's shapes hold and where they do not (profiles/planner_coverage_map.md)."""
+    import torch
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    from paper_2211_00889_b200 import workloads as WL
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peak()
+    base = WL.WORKLOADS[DEFAULT_WORKLOAD]
+    cells = []
+    for variant, topology in (("dpsgd", "ring"), ("allreduce", "full"), ("centralized", "full")):
+        for order in ("mix_then_update", "update_then_mix"):
+            if variant == "centralized" and order != "mix_then_update":
+                continue
+            for dtype in ("bf16", "f32"):
+                es = 2 if dtype == "bf16" else 4
+                for K in (1, 2, 4, 8, 16, 32, 64):
+                    for M in (1, 2, 4, 8, 16):
+                        P = int(min(base.P, 5e9 / (K * M * es), 8e9 / (K * 16)))
+                        P -= P % 512
+                        w = replace(base, K=K, M=M, P=P, grad_dtype=dtype, variant=variant, topology=topology,
+                                    name="K%d_M%d" % (K, M))
+                        r = Runner(B, WL, w, dev, order=order)
+                        res = r.timed("fused", 10, 3, sampler=ClockSampler(0))
+                        gbs = sum(res["alg_bytes"]) / 10 / (res["launch_ms"] * 1e-3) / 1e9
+                        cells.append({"variant": variant, "topology": topology, "order": order, "grad_dtype": dtype,
+                                      "K": K, "M": M, "P": P, "ms_per_step": res["launch_ms"], "achieved_hbm_gbs": gbs,
+                                      "frac": gbs / peak, "kernel_plan": res["kernel_plan"]})
+                        r.close()
+                        del r
+                        torch.cuda.empty_cache()
+    print(json.dumps({"coverage_map": cells, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s"}))
+
+
 def main():
     args = parse_args()
     from paper_2211_00889_b200 import workloads as WL
+    if args.coverage_map:
+        return coverage_map(args)
     w = WL.WORKLOADS[args.workload]
     if args.cols:
         w = replace(WL.scaled(w, args.cols), name="%s[P=%d]" % (w.name, args.cols))
