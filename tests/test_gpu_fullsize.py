@@ -150,6 +150,37 @@ def test_mid_size_every_column_update_then_mix():
     ctx.close()
 
 
+@pytest.mark.parametrize("K,M,order", [(2, 2, "mix_then_update"), (3, 8, "mix_then_update"), (5, 3, "update_then_mix")])
+def test_mid_size_every_column_few_learners(K, M, order):
+    """Few learners run four CTAs per SM of one consumer group each; 2400 tiles give every CTA four or
+    more of them, and every column is compared with the oracle."""
+    import torch
+    from dataclasses import replace
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    w = replace(WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 2400 * 512 + 24, steps=3), K=K, M=M)
+    ctx = B.context_for(w)
+    if order == "update_then_mix":
+        ctx.set_option(B.NB_OPT_ORDER, B.NB_ORDER_UPDATE_THEN_MIX)
+    orc = H.oracle_for(w, w.P, order=order)
+    x0 = WL.init_params(w)
+    ctx.set_params(torch.from_numpy(x0).cuda())
+    orc.set_params(x0)
+    for t in range(w.steps):
+        n = H.lib_counts(B, w, t)
+        payload, values = WL.gradients_np(w, t)
+        ctx.step_fused(H.to_device(payload), n)
+        orc.step(values, n.tolist())
+        del payload, values
+    plan = ctx.get_kernel_plan()
+    assert plan["pipeline"] == 1 and plan["groups"] == 1 and plan["tiles"] >= 4 * plan["grid"]
+    H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT, "X")
+    H.assert_close(ctx.get_momentum().numpy(), orc.V, H.TOL_SAME_INPUT, "V")
+    ctx.check_guards()
+    ctx.close()
+
+
 def test_more_than_two_to_the_31_columns():
     """Column indices beyond 32 bits: one learner pair, 2^31 + 1544 columns (the last window the
     oracle checks lies entirely above 2^31)."""
