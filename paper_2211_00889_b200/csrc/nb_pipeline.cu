@@ -881,7 +881,8 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   static const Shape small_item_shapes[] = {{512, 1, 4, 2, 8}, {512, 2, 2, 2, 8}, {512, 1, 4, 1, 8}, {512, 1, 4, 1, 4},
                                             {256, 1, 4, 2, 8}, {128, 1, 4, 2, 8}};
   const bool mix_first = a.order == NB_ORDER_MIX_THEN_UPDATE;
-  const bool small_items = mix_first && slot_bytes_of(512 * 4, 512, es, Rmax, row_pad) <= 6400;  // <= 4 bf16 / 2 fp32 rows
+  const bool small_slot = slot_bytes_of(512 * 4, 512, es, Rmax, row_pad) <= 6400;  // <= 4 bf16 / 2 fp32 rows
+  const bool small_items = mix_first && small_slot;
   // Rows named by a pointer table (the streaming entry points in hold mode) also do best on one CTA per SM
   // with four groups (cfg3 sizes: 0.99 against 0.98 for two CTAs of two groups).
   const bool one_cta_first = small_items || (mix_first && a.row_ptrs != nullptr);
@@ -896,7 +897,6 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   // Update-then-mix, K <= 8 (before: K = 2 0.37-0.55, K = 4 0.64-0.88, K = 6 0.64-0.86): four such CTAs, with three X
   // buffers for K <= 2 and small items (K = 2 0.74-0.94, K = 4 0.84-1.00); K = 6, 7 with 8-row items two CTAs of two
   // groups (0.86 -> 1.02); K = 8 with 8-row items keeps the table (1.02).
-  const bool small_slot = slot_bytes_of(512 * 4, 512, es, Rmax, row_pad) <= 6400;
   Shape first = {0, 0, 0, 0, 0};
   if (!a.row_ptrs) {
     if (mix_first) {
@@ -914,8 +914,7 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   // The update-then-mix order releases no slot while a group averages, so its ring is what keeps memory busy: a shape is
   // taken there only if the rings of an SM hold at least 56 KB (K = 32, M = 1: three X buffers leave 8 slots of 3 KB,
   // 0.77; two leave 32, 0.96.  K = 40, M = 4: two buffers with 8 slots of 6 KB 0.81, one buffer with 24 0.90; K = 40,
-  // M = 1: two buffers with 20 slots of 3 KB 1.00); if no
-  // shape offers that, the first one that fits at all.
+  // M = 1: two buffers with 20 slots of 3 KB 1.00); if no shape offers that, the first one that fits at all.
   struct Chosen { int T, ctas, groups, slots, x_stages, R; };
   Chosen c = {0, 0, 0, 0, 0, 0}, fallback = {0, 0, 0, 0, 0, 0};
   for (int q = 0; q < n_shapes && !c.T; ++q) {
