@@ -277,7 +277,11 @@ int nb_get_finished(const nb_ctx *c, int32_t *finished /* host out [K] */, int32
 int nb_step(nb_ctx *c, void *stream);
 
 /* Steps 1-4 in a single pass over the gradient stream without the acc round trip.  The result is
- * bit-identical to nb_accumulate followed by nb_step.  Arguments as nb_accumulate. */
+ * bit-identical to nb_accumulate followed by nb_step.  Arguments as nb_accumulate.
+ * CUDA graphs: nb_accumulate, nb_step and nb_step_fused only enqueue kernels on `stream` (no
+ * allocation, copy or synchronisation), so they may be called while `stream` is being captured;
+ * the finished counts, the pointers and (MATCHA) the step index are fixed in the captured launches,
+ * and the host-side step counter advances once per call, not per replay. */
 int nb_step_fused(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
                   const int32_t *finished, void *stream);
 

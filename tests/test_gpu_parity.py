@@ -586,6 +586,43 @@ def test_work_is_enqueued_on_the_callers_stream(B):
     ref.close(); other.close()
 
 
+@pytest.mark.parametrize("fused", [True, False])
+def test_step_can_be_captured_in_a_cuda_graph(B, fused):
+    """The step entry points only enqueue kernels on the caller's stream (no allocation, copy or
+    synchronisation once a context has run its first step), so an iteration can be captured in a CUDA
+    graph and replayed: three replays equal three plain calls bit for bit."""
+    import torch
+    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 9 * 512 + 40, steps=4)
+    x0 = torch.from_numpy(WL.init_params(w)).cuda()
+    G = H.to_device(WL.gradients_np(w, 0)[0])
+    n = H.lib_counts(B, w, 0)
+    plain, graphed = B.context_for(w), B.context_for(w)
+
+    def step(ctx):
+        if fused:
+            ctx.step_fused(G, n)
+        else:
+            ctx.accumulate(G, n)
+            ctx.step()
+
+    for ctx in (plain, graphed):
+        ctx.set_params(x0)
+        step(ctx)                                  # first step outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step(graphed)                              # recorded, not run
+    for _ in range(3):
+        graph.replay()
+        step(plain)
+    torch.cuda.synchronize()
+    assert torch.equal(graphed.get_params(device="cuda"), plain.get_params(device="cuda"))
+    assert torch.equal(graphed.get_momentum(device="cuda"), plain.get_momentum(device="cuda"))
+    graphed.check_guards()
+    del graph
+    plain.close(); graphed.close()
+
+
 @pytest.mark.parametrize("name", ["cfg2_allreduce_resnet18", "cfg3_dpsgd_ring_resnet50", "cfg4_matcha_vgg16",
                                   "cfg5_scale_ring"])
 def test_full_step_counts_of_the_configurations(B, name):
