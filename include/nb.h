@@ -281,7 +281,8 @@ int nb_step(nb_ctx *c, void *stream);
  * CUDA graphs: nb_accumulate, nb_step and nb_step_fused only enqueue kernels on `stream` (no
  * allocation, copy or synchronisation), so they may be called while `stream` is being captured;
  * the finished counts, the pointers and (MATCHA) the step index are fixed in the captured launches,
- * and the host-side step counter advances once per call, not per replay. */
+ * and the host-side step counter advances once per call, not per replay.  (Not nb_step after
+ * deliveries in NB_STREAMING_HOLD mode: it uploads the table of delivered vectors first.) */
 int nb_step_fused(nb_ctx *c, const void *grads, int dtype, int64_t ld_m, int64_t ld_k,
                   const int32_t *finished, void *stream);
 
