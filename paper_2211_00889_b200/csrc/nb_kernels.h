@@ -64,6 +64,7 @@ struct PipePlan {
   int row_copies;  // 0: gradient rows travel as tensor-map boxes; 1: one bulk copy per row (rows not 16-byte aligned);
                    // 2: one bulk copy per row from a table of row pointers
   int x_stages;    // buffers of the step kernel's X stage (0 for the kernels that have none)
+  bool x_in_ring = false;  // step kernel, update-then-mix on one buffer: old model rows travel in the ring items
   int quads_per_thread = 1;  // groups of four columns per consumer thread (no-stage kernels: 1 or 2)
 };
 bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan);

@@ -165,8 +165,10 @@ struct PipeArgs {
   const unsigned char *g_base;
   int64_t g_ld_m_bytes, g_ld_k_bytes;
   int32_t g_mis0, g_mis_m, g_mis_k;
+  int32_t x_in_ring;  // update-then-mix on one buffer: the old model row of a learner travels in its ring item
   alignas(64) CUtensorMap xmap;                   // X as [K, units]: box = (256, K)
   alignas(64) CUtensorMap vmap;                   // V as [K, units]: box = (256, 1)
+  alignas(64) CUtensorMap xrmap;                  // X as [K, units]: box = (256, 1) (x_in_ring only)
   alignas(64) CUtensorMap gmap[kMaxRowsPerItem];  // G as [K, M, units]: box = (256, r, 1), r = 1..R
 };
 
@@ -337,8 +339,9 @@ struct PipeLayout {
 
 // row_pad: 0 for box copies, 16 when every row is staged as its 16-byte aligned superset.
 constexpr int kMaxXStages = 3;
+// state_rows: fp32 state rows at the head of a slot (1: the momentum row; 2: momentum row and old model row).
 __host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, int n_slots, int mix_slots, int row_pad,
-                                                  int x_stages) {
+                                                  int x_stages, int state_rows = 1) {
   PipeLayout L;
   int off = (2 * n_slots + 3 * kMaxXStages) * 8;
   off = (off + 127) / 128 * 128;
@@ -348,7 +351,7 @@ __host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, i
   L.off_xs = off;
   off += x_stages * K * T * 4;  // two buffers: tile t+1's models load while tile t is consumed (see the kernel)
   L.off_slots = off;
-  L.slot_bytes = slot_bytes_of(T * 4, T, es, R, row_pad);
+  L.slot_bytes = slot_bytes_of(T * 4 * state_rows, T, es, R, row_pad);
   L.total = off + n_slots * L.slot_bytes;
   return L;
 }
@@ -367,7 +370,12 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
   const int K = s.K, T = TT ? TT : a.T, R = a.rows_per_item, NS = a.n_slots, NG = a.n_groups;
   const int NSG = NS / NG;  // slots in each group's ring
   const int NXS = a.x_stages;
-  const PipeLayout L = pipe_layout(K, T, ES, R, NS, s.mix_slots, kRowPad, NXS);
+  // Update-then-mix on ONE buffer (K > 32): the old model row x_i rides in learner i's ring item next to v_i, the
+  // consumers write y_i = x_i - lr v_i into the buffer themselves, and nobody has to wait for a [K, T] box of old
+  // models between two tiles: the ring keeps bringing the next tile's items while this tile is averaged.
+  const bool xr = a.x_in_ring != 0;
+  const int state_bytes = T * 4 * (xr ? 2 : 1);  // fp32 state rows at the head of a slot
+  const PipeLayout L = pipe_layout(K, T, ES, R, NS, s.mix_slots, kRowPad, NXS, xr ? 2 : 1);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);
   uint64_t *empty = full + NS;
   uint64_t *xfull = empty + NS;
@@ -443,11 +451,14 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
             }
             unsigned char *dst = slots + (size_t)sl * L.slot_bytes;
             if (lane == 0) {
-              mbar_expect_tx(&full[sl], (uint32_t)(rows * (T * ES + kRowPad) + (m0 == 0 ? T * 4 : 0)));
-              if (m0 == 0) tma_load_2d(dst, &a.vmap, tile * kBoxInner, i, &full[sl]);
+              mbar_expect_tx(&full[sl], (uint32_t)(rows * (T * ES + kRowPad) + (m0 == 0 ? state_bytes : 0)));
+              if (m0 == 0) {
+                tma_load_2d(dst, &a.vmap, tile * kBoxInner, i, &full[sl]);
+                if (xr) tma_load_2d(dst + T * 4, &a.xrmap, tile * kBoxInner, i, &full[sl]);
+              }
             }
             if constexpr (kWarpIssue) __syncwarp();
-            issue_rows<ES, GM>(a, dst + T * 4, T, tile, i, m0, rows, lane, &full[sl]);
+            issue_rows<ES, GM>(a, dst + state_bytes, T, tile, i, m0, rows, lane, &full[sl]);
             if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
             m0 += R;
           } while (m0 < n);
@@ -460,7 +471,7 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
     // release, so with two buffers tile t+1's models load while tile t is consumed.  (One buffer:
     // K so large that two do not fit; the ring keeps filling while the next tile's models load.
     // Three: the update-then-mix order, whose averaging pass runs one tile late.)
-    if (lane == 0) {
+    if (lane == 0 && !xr) {
       int titer = 0, b = 0;
       uint32_t xpar = 0;
       for (int tile = blockIdx.x; ok && tile < a.n_tiles; tile += gridDim.x, ++titer) {
@@ -529,7 +540,8 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
         float *Vc = s.V + col0;
         float4 *xs4w = reinterpret_cast<float4 *>(xs_base + (size_t)xb * K * T);
         const float4 *xs4 = xs4w;
-        ok = __all_sync(0xffffffffu, mbar_wait(&xfull[xb], xpar, a.err, 3));  // warp-uniform outcome
+        // the tile's old models are staged; x_in_ring: the buffer is free (every group has averaged the previous tile)
+        ok = __all_sync(0xffffffffu, xr ? mbar_wait(&xempty[xb], xpar ^ 1, a.err, 3) : mbar_wait(&xfull[xb], xpar, a.err, 3));
         if (!ok) break;
         if constexpr (kDebug) {  // this thread's stores of the tile: 4 columns of all K rows of X and V
           ok = __all_sync(0xffffffffu,
@@ -551,7 +563,7 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
           }
           const int n = s.n[i];
           float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f), xi = v;
           int m0 = 0;
           do {
             const int rows = (n - m0 < R) ? (n - m0) : R;
@@ -564,9 +576,12 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
               if (!ok) break;
             }
             const unsigned char *src = slots + (size_t)sl * L.slot_bytes;
-            if (m0 == 0) v = reinterpret_cast<const float4 *>(src)[cq];
+            if (m0 == 0) {
+              v = reinterpret_cast<const float4 *>(src)[cq];
+              if (xr) xi = reinterpret_cast<const float4 *>(src + T * 4)[cq];
+            }
             const int s0 = GA ? 0 : (a.g_mis0 + i * a.g_mis_k + m0 * a.g_mis_m);
-            acc = sum_rows<SRC, GA>(acc, src + T * 4 + cq * 4 * ES, T * ES + kRowPad, rows, s0, a.g_mis_m);
+            acc = sum_rows<SRC, GA>(acc, src + state_bytes + cq * 4 * ES, T * ES + kRowPad, rows, s0, a.g_mis_m);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[sl]);
             if (++slot == (uint32_t)NSG) { slot = 0; phase ^= 1; }
@@ -581,7 +596,7 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
             else xh = mix_row(xs4, nq, cq, s_col, s_val, s_beg[i], s_end[i]);
             st4(Xc + (int64_t)i * ldx, descend(xh, lr, vn));
           } else {
-            xs4w[i * nq + cq] = descend(xs4[i * nq + cq], lr, vn);  // y_i replaces x_i in the buffer
+            xs4w[i * nq + cq] = descend(xr ? xi : xs4[i * nq + cq], lr, vn);  // y_i replaces x_i in the buffer
           }
         }
         if (!ok) break;
@@ -798,7 +813,7 @@ __global__ void nb_wait_selftest_kernel(int *err, int code, long long limit_cycl
 }
 
 struct PipeTuning {
-  int T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0, x_stages = 0, qpt = 0;
+  int T = 0, slots = 0, ctas_per_sm = 0, rows = 0, groups = 0, x_stages = 0, qpt = 0, xr = -1;
   int sm_count = 0;
 };
 
@@ -819,6 +834,7 @@ PipeTuning &tuning() {
     q.groups = geti("NB_PIPELINE_GROUPS", 0);
     q.x_stages = geti("NB_PIPELINE_XSTAGES", 0);
     q.qpt = geti("NB_PIPELINE_QPT", 0);
+    q.xr = geti("NB_PIPELINE_XR", -1);
 #endif
     return q;
   }();
@@ -934,11 +950,12 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   // halves the rows per ring item (the slots shrink) so that 512-column tiles still fit where 8-row
   // items do not (K = 64 with fp32 gradients: 0.94 on 256-column tiles).  A tuning build's overrides
   // replace the corresponding field of every shape.
-  struct Shape { int T, ctas, groups, x_stages, rows; };
+  struct Shape { int T, ctas, groups, x_stages, rows, xr = 0; };  // xr: old model rows travel in the ring items
   static const Shape mix_first_shapes[] = {{512, 2, 2, 2, 8}, {512, 1, 4, 2, 8}, {512, 1, 4, 1, 8}, {512, 1, 4, 1, 4},
                                            {256, 1, 4, 2, 8}, {128, 1, 4, 2, 8}};
-  static const Shape update_first_shapes[] = {{512, 1, 4, 3, 8}, {512, 2, 2, 2, 8}, {512, 1, 4, 2, 8}, {512, 1, 4, 1, 8},
-                                              {512, 1, 4, 1, 4}, {256, 1, 4, 2, 8}, {128, 1, 4, 2, 8}};
+  static const Shape update_first_shapes[] = {{512, 1, 4, 3, 8}, {512, 2, 2, 2, 8}, {512, 1, 4, 2, 8}, {512, 1, 4, 1, 8, 1},
+                                              {512, 1, 4, 1, 8}, {512, 1, 4, 1, 4, 1}, {512, 1, 4, 1, 4}, {256, 1, 4, 2, 8},
+                                              {128, 1, 4, 2, 8}};
   // Few mini-batches per batch (items of a momentum row and at most 4 KB of gradient rows): one CTA
   // per SM with four groups and three slots per group (cfg4 sizes at P = 138M: 0.99 of the measured
   // copy bandwidth against 0.95 for two CTAs with two groups of two slots; equal within 1 % at 25-51M).
@@ -971,16 +988,16 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
       else if (a.K <= 7) first = {512, 2, 2, 2, 8};
     }
   }
-  Shape shapes[8];
+  Shape shapes[10];
   int n_shapes = 0;
   if (first.T) shapes[n_shapes++] = first;
-  for (int q = 0; q < (mix_first ? 6 : 7); ++q) shapes[n_shapes++] = table[q];
+  for (int q = 0; q < (mix_first ? 6 : 9); ++q) shapes[n_shapes++] = table[q];
   // The update-then-mix order releases no slot while a group averages, so its ring is what keeps memory busy: a shape is
   // taken there only if the rings of an SM hold at least 56 KB (K = 32, M = 1: three X buffers leave 8 slots of 3 KB,
   // 0.77; two leave 32, 0.96.  K = 40, M = 4: two buffers with 8 slots of 6 KB 0.81, one buffer with 24 0.90; K = 40,
   // M = 1: two buffers with 20 slots of 3 KB 1.00); if no shape offers that, the first one that fits at all.
-  struct Chosen { int T, ctas, groups, slots, x_stages, R; };
-  Chosen c = {0, 0, 0, 0, 0, 0}, fallback = {0, 0, 0, 0, 0, 0};
+  struct Chosen { int T, ctas, groups, slots, x_stages, R, xr; };
+  Chosen c = {0, 0, 0, 0, 0, 0, 0}, fallback = {0, 0, 0, 0, 0, 0, 0};
   for (int q = 0; q < n_shapes && !c.T; ++q) {
     const Shape &sh = shapes[q];
     Chosen k;
@@ -989,20 +1006,24 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
     k.ctas = t.ctas_per_sm ? t.ctas_per_sm : sh.ctas;
     k.groups = t.groups ? t.groups : sh.groups;
     k.x_stages = t.x_stages ? t.x_stages : sh.x_stages;
+    k.xr = (!mix_first && k.x_stages == 1 && sh.xr && t.xr != 0) ? 1 : 0;
     if (k.T != 128 && k.T != 256 && k.T != 512) return false;
     if (k.x_stages < 1 || k.x_stages > kMaxXStages) return false;
     if (k.groups > kMaxGroups) k.groups = kMaxGroups;
     if (k.groups > a.K) k.groups = a.K;
     while (k.groups > 1 && k.groups * (k.T / 4) > 512) --k.groups;
     if (k.groups < 1 || k.ctas < 1) return false;
-    const PipeLayout L0 = pipe_layout(a.K, k.T, es, k.R, 0, a.mix_slots, row_pad, k.x_stages);
+    const PipeLayout L0 = pipe_layout(a.K, k.T, es, k.R, 0, a.mix_slots, row_pad, k.x_stages, 1 + k.xr);
     const int budget = kSmemBudget / k.ctas - 1024;
-    const int slot_bytes = slot_bytes_of(k.T * 4, k.T, es, k.R, row_pad);
+    const int slot_bytes = L0.slot_bytes;
     k.slots = (budget - L0.total - 256) / slot_bytes;
     if (t.slots && t.slots < k.slots) k.slots = t.slots;
     if (k.slots > 32) k.slots = 32;
     k.slots -= k.slots % k.groups;  // every group's ring has the same number of slots
     if (k.slots < 2 * k.groups) continue;
+    // old models in the ring: only with three slots per group (K = 48, bf16: M = 4, 16 slots 0.84 -> 0.97; M = 8, 8 slots
+    // 0.94 -> 0.90: with two slots per group the larger items starve the ring, and the plain one-buffer shape follows)
+    if (k.xr && k.slots < 3 * k.groups) continue;
     if (!fallback.T) fallback = k;
     // Alg. 2 order, learners that need several items per tile (M > R): two CTAs per SM are taken only with four slots
     // per group (K = 16, M = 16, bf16: two slots per group 0.99, one CTA of four groups with every slot that fits 1.03).
@@ -1012,7 +1033,7 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   }
   if (!c.T) c = fallback;
   if (!c.T) return false;
-  const int T = c.T, ctas = c.ctas, groups = c.groups, x_stages = c.x_stages, R = c.R;
+  const int T = c.T, ctas = c.ctas, groups = c.groups, x_stages = c.x_stages, R = c.R, xr = c.xr;
   int slots = c.slots;
   const Coverage cov = coverage(a, es, T);
   if (cov.n_tiles < 1) return false;
@@ -1028,7 +1049,7 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   // group averages: cfg3 sizes 12 slots 1.04, 8 slots 0.99).
   const int per_group = (small_items && ctas == 1) ? 3 : 2;
   if (!t.slots && mix_first && x_stages == 2 && R >= a.M && slots > per_group * groups) slots = per_group * groups;
-  const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots, row_pad, x_stages);
+  const PipeLayout L = pipe_layout(a.K, T, es, R, slots, a.mix_slots, row_pad, x_stages, 1 + xr);
   if (L.total > kSmemBudget) return false;
   plan->T = T;
   plan->rows_per_item = R;
@@ -1039,6 +1060,7 @@ bool plan_pipeline(const StepArgs &a, int es, PipePlan *plan) {
   plan->head = (int)cov.head;
   plan->row_copies = a.row_ptrs ? 2 : rows_aligned ? 0 : 1;
   plan->x_stages = x_stages;
+  plan->x_in_ring = xr != 0;
   const int64_t max_ctas = (int64_t)ctas * t.sm_count;
   plan->grid = (int)(plan->n_tiles < max_ctas ? plan->n_tiles : max_ctas);
   return true;
@@ -1129,6 +1151,7 @@ void fill_pipe_args(PipeArgs *p, const StepArgs &a, const PipePlan &plan, int *e
   p->n_tiles = plan.n_tiles;
   p->n_groups = plan.n_groups;
   p->x_stages = plan.x_stages;
+  p->x_in_ring = plan.x_in_ring ? 1 : 0;
   p->err = err_flag;
 }
 }  // namespace
@@ -1202,7 +1225,8 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
     const cuuint64_t strides[1] = {(cuuint64_t)a.ldx * 4};
     const cuuint32_t xbox[2] = {kBoxInner, (cuuint32_t)a.K};
     const cuuint32_t vbox[2] = {kBoxInner, 1};
-    if (!encode_map(&p.xmap, a.X, ub, 2, dims, strides, xbox) || !encode_map(&p.vmap, a.V, ub, 2, dims, strides, vbox))
+    if (!encode_map(&p.xmap, a.X, ub, 2, dims, strides, xbox) || !encode_map(&p.vmap, a.V, ub, 2, dims, strides, vbox) ||
+        (plan.x_in_ring && !encode_map(&p.xrmap, a.X, ub, 2, dims, strides, vbox)))
       return cudaErrorNotSupported;  // nothing launched: caller falls back to the direct-load kernel
   }
   if (plan.row_copies == 1) fill_row_args(&p, a, es);
