@@ -123,13 +123,17 @@ def test_mid_size_every_column_centralized(dtype, tiles):
         c.close()
 
 
-def test_mid_size_every_column_update_then_mix():
-    """Eq. 4-6's order on 1200 tiles: the deferred averaging pass over three X buffers, every column."""
+@pytest.mark.parametrize("K,M,tiles,x_buffers", [(16, 8, 1200, 3), (32, 8, 600, 2), (40, 4, 600, 1)])
+def test_mid_size_every_column_update_then_mix(K, M, tiles, x_buffers):
+    """Eq. 4-6's order on several tiles per CTA, every column: the deferred averaging pass over three X
+    buffers (K = 16), the half-deferred pass over two (K = 32), and the single buffer whose old model
+    rows travel in the ring items (K = 40)."""
     import torch
+    from dataclasses import replace
     from paper_2211_00889_b200.build import build_library
     build_library()
     from paper_2211_00889_b200 import binding as B
-    w = WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], 1200 * 512 + 24, steps=3)
+    w = replace(WL.scaled(WL.WORKLOADS["cfg3_dpsgd_ring_resnet50"], tiles * 512 + 24, steps=3), K=K, M=M)
     ctx = B.context_for(w)
     ctx.set_option(B.NB_OPT_ORDER, B.NB_ORDER_UPDATE_THEN_MIX)
     orc = H.oracle_for(w, w.P, order="update_then_mix")
@@ -143,7 +147,7 @@ def test_mid_size_every_column_update_then_mix():
         orc.step(values, n.tolist())
         del payload, values
     plan = ctx.get_kernel_plan()
-    assert plan["pipeline"] == 1 and plan["x_buffers"] == 3 and plan["tiles"] >= 3 * plan["grid"]
+    assert plan["pipeline"] == 1 and plan["x_buffers"] == x_buffers and plan["tiles"] >= 3 * plan["grid"]
     H.assert_close(ctx.get_params().numpy(), orc.X, H.TOL_SAME_INPUT, "X")
     H.assert_close(ctx.get_momentum().numpy(), orc.V, H.TOL_SAME_INPUT, "V")
     ctx.check_guards()
