@@ -165,10 +165,9 @@ struct PipeArgs {
   const unsigned char *g_base;
   int64_t g_ld_m_bytes, g_ld_k_bytes;
   int32_t g_mis0, g_mis_m, g_mis_k;
-  int32_t x_in_ring;  // update-then-mix on one buffer: the old model row of a learner travels in its ring item
   alignas(64) CUtensorMap xmap;                   // X as [K, units]: box = (256, K)
   alignas(64) CUtensorMap vmap;                   // V as [K, units]: box = (256, 1)
-  alignas(64) CUtensorMap xrmap;                  // X as [K, units]: box = (256, 1) (x_in_ring only)
+  alignas(64) CUtensorMap xrmap;                  // X as [K, units]: box = (256, 1) (template parameter XR only)
   alignas(64) CUtensorMap gmap[kMaxRowsPerItem];  // G as [K, M, units]: box = (256, r, 1), r = 1..R
 };
 
@@ -359,7 +358,8 @@ __host__ __device__ inline PipeLayout pipe_layout(int K, int T, int es, int R, i
 // ES = bytes per gradient element (2: bf16, 4: fp32).
 // TT = tile width known at compile time (512, the usual shape: strides become immediates) or 0 (a.T).
 // GM = how the gradient rows travel: kGBox, kGRows or kGPtrs (see above).
-template <int ES, bool MEAN, int TT, int GM>
+// XR = the old model rows travel in the ring items (update-then-mix on one buffer; see below).
+template <int ES, bool MEAN, int TT, int GM, bool XR = false>
 __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeline_kernel(const __grid_constant__ PipeArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int SRC = ES == 2 ? kSrcBF16 : kSrcF32;
@@ -373,7 +373,7 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
   // Update-then-mix on ONE buffer (K > 32): the old model row x_i rides in learner i's ring item next to v_i, the
   // consumers write y_i = x_i - lr v_i into the buffer themselves, and nobody has to wait for a [K, T] box of old
   // models between two tiles: the ring keeps bringing the next tile's items while this tile is averaged.
-  const bool xr = a.x_in_ring != 0;
+  constexpr bool xr = XR;
   const int state_bytes = T * 4 * (xr ? 2 : 1);  // fp32 state rows at the head of a slot
   const PipeLayout L = pipe_layout(K, T, ES, R, NS, s.mix_slots, kRowPad, NXS, xr ? 2 : 1);
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);
@@ -540,7 +540,7 @@ __global__ void __launch_bounds__((kMaxGroups + 1) * 32 + 512, 1) nb_step_pipeli
         float *Vc = s.V + col0;
         float4 *xs4w = reinterpret_cast<float4 *>(xs_base + (size_t)xb * K * T);
         const float4 *xs4 = xs4w;
-        // the tile's old models are staged; x_in_ring: the buffer is free (every group has averaged the previous tile)
+        // the tile's old models are staged; XR: the buffer is free (every group has averaged the previous tile)
         ok = __all_sync(0xffffffffu, xr ? mbar_wait(&xempty[xb], xpar ^ 1, a.err, 3) : mbar_wait(&xfull[xb], xpar, a.err, 3));
         if (!ok) break;
         if constexpr (kDebug) {  // this thread's stores of the tile: 4 columns of all K rows of X and V
@@ -1151,7 +1151,6 @@ void fill_pipe_args(PipeArgs *p, const StepArgs &a, const PipePlan &plan, int *e
   p->n_tiles = plan.n_tiles;
   p->n_groups = plan.n_groups;
   p->x_stages = plan.x_stages;
-  p->x_in_ring = plan.x_in_ring ? 1 : 0;
   p->err = err_flag;
 }
 }  // namespace
@@ -1201,7 +1200,9 @@ cudaError_t configure_pipeline() {
 #define NB_CFG(ES, MEAN)                                                                                         \
   NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGBox>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, kGBox>)     \
   NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGRows>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, kGRows>)   \
-  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGPtrs>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, kGPtrs>)
+  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGPtrs>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 0, kGPtrs>)   \
+  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGBox, true>) NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGRows, true>) \
+  NB_CFG1(nb_step_pipeline_kernel<ES, MEAN, 512, kGPtrs, true>)
   NB_CFG(2, true) NB_CFG(2, false) NB_CFG(4, true) NB_CFG(4, false)
 #undef NB_CFG
 #define NB_CFG(ES, MODE)                                                                                            \
@@ -1238,10 +1239,17 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
     else if (plan.row_copies == 1) nb_step_pipeline_kernel<ES, MEAN, TT, kGRows><<<plan.grid, threads, plan.smem_bytes, st>>>(p); \
     else nb_step_pipeline_kernel<ES, MEAN, TT, kGBox><<<plan.grid, threads, plan.smem_bytes, st>>>(p);                            \
   } while (0)
-#define NB_LAUNCH(ES, MEAN)                       \
-  do {                                            \
-    if (plan.T == 512) NB_LAUNCH2(ES, MEAN, 512); \
-    else NB_LAUNCH2(ES, MEAN, 0);                 \
+#define NB_LAUNCH_XR(ES, MEAN)                                                                                          \
+  do {                                                                                                                  \
+    if (plan.row_copies == 2) nb_step_pipeline_kernel<ES, MEAN, 512, kGPtrs, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);      \
+    else if (plan.row_copies == 1) nb_step_pipeline_kernel<ES, MEAN, 512, kGRows, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p); \
+    else nb_step_pipeline_kernel<ES, MEAN, 512, kGBox, true><<<plan.grid, threads, plan.smem_bytes, st>>>(p);                            \
+  } while (0)
+#define NB_LAUNCH(ES, MEAN)                                          \
+  do {                                                               \
+    if (plan.x_in_ring && plan.T == 512) NB_LAUNCH_XR(ES, MEAN);     \
+    else if (plan.T == 512) NB_LAUNCH2(ES, MEAN, 512);               \
+    else NB_LAUNCH2(ES, MEAN, 0);                                    \
   } while (0)
   if (es == 2) {
     if (a.mean_mode) NB_LAUNCH(2, true);
@@ -1251,6 +1259,7 @@ cudaError_t launch_step_pipeline(const StepArgs &a, int es, const PipePlan &plan
     else NB_LAUNCH(4, false);
   }
 #undef NB_LAUNCH
+#undef NB_LAUNCH_XR
 #undef NB_LAUNCH2
   return cudaGetLastError();
 }
