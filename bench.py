@@ -51,7 +51,7 @@ TRAFFIC_PER_ALGORITHMIC_BYTE = {
     "cfg3_dpsgd_ring_resnet50[streaming_hold]": 0.988,
     "cfg3_dpsgd_ring_resnet50[centralized]": 0.996,
     "cfg2_allreduce_resnet18": 0.990,
-    "cfg4_matcha_vgg16": 0.981,
+    "cfg4_matcha_vgg16": 0.980,
     "cfg5_scale_allreduce": 0.990,
     "cfg5_scale_ring": 0.990,
     "ring_K64_P12.8M": 0.987,
