@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 # columns).  No entry: no capture exists and `traffic` is reported as null.
 TRAFFIC_PER_ALGORITHMIC_BYTE = {
     "cfg3_dpsgd_ring_resnet50": 0.988,
-    "cfg3_dpsgd_ring_resnet50[P+1, rows not 16-byte aligned]": 0.988,
+    "cfg3_dpsgd_ring_resnet50[P+1, rows not 16-byte aligned]": 0.989,
     "cfg3_dpsgd_ring_resnet50[update_then_mix]": 0.987,
     "cfg3_dpsgd_ring_resnet50[unfused]": 1.283,
     "cfg3_dpsgd_ring_resnet50[streaming_hold]": 0.988,
