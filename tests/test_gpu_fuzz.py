@@ -157,3 +157,67 @@ def test_random_differential_between_kernel_families(case_id):
     assert torch.equal(a.get_momentum(), d.get_momentum()), case
     a.check_guards(); d.check_guards()
     a.close(); d.close()
+
+
+@pytest.mark.parametrize("case_id", range(24))
+def test_random_differential_with_many_tiles_per_cta(case_id):
+    """The differential test in the persistent regime: about 4100 tiles, so that every CTA of every
+    kernel shape (up to nine CTAs per SM) takes three or more tiles - ring phases wrap, X buffers are
+    reused, the old-models-in-the-ring buffer is handed on from tile to tile - and the default kernels
+    must still give the bits of the direct-load kernels."""
+    import torch
+    from paper_2211_00889_b200.build import build_library
+    build_library()
+    from paper_2211_00889_b200 import binding as B
+    rng = np.random.default_rng(77000 + case_id)
+    variant = str(rng.choice(["allreduce", "ring", "matcha", "centralized"]))
+    K = int(rng.choice([1, 2, 3, 5, 8, 16, 24, 33, 40, 48, 64])) if variant != "matcha" else int(rng.choice([4, 8, 16, 24]))
+    M = int(rng.integers(1, 7 if K >= 33 else 13))
+    P = 512 * int(rng.integers(4100, 4300)) + int(rng.choice([0, 8, rng.integers(1, 512)]))
+    dtype = torch.bfloat16 if rng.integers(0, 2) else torch.float32
+    order = int(rng.integers(0, 2))
+    shift = int(rng.choice([0, 0, 1]))
+    fused = bool(rng.integers(0, 2))
+    seed = int(rng.integers(0, 2 ** 40))
+
+    def make():
+        if variant == "allreduce":
+            return B.NbContext(K, P, M, 0.05, 0.9, "allreduce")
+        if variant == "ring":
+            return B.NbContext(K, P, M, 0.05, 0.9, "dpsgd", B.make_topology("ring"))
+        if variant == "matcha":
+            topo = B.make_topology("random_regular", degree=3 if K > 4 else 2, seed=seed, alpha=0.2, act_prob=0.6)
+            return B.NbContext(K, P, M, 0.05, 0.9, "matcha", topo)
+        return B.NbContext(K, P, M, 0.05, 0.9, "centralized")
+
+    a, d = make(), make()
+    d.set_option(B.NB_OPT_KERNEL, B.NB_KERNEL_DIRECT)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    x0 = torch.randn(P, generator=gen, device="cuda") * 0.01
+    for c in (a, d):
+        if variant != "centralized":
+            c.set_option(B.NB_OPT_ORDER, order)
+        c.set_params(x0)
+    flat = torch.empty(K * M * P + shift, dtype=dtype, device="cuda")
+    g = flat[shift:].view(K, M, P)                       # `shift` elements off the allocation's 16-byte boundary
+    plan = None
+    for t in range(3):
+        for i in range(K):                               # drawn learner by learner: no fp32 copy of the whole stream
+            g[i].copy_(torch.randn((M, P), generator=gen, device="cuda") * 0.01)
+        n = rng.integers(0, M + 1, K)
+        for c in (a, d):
+            if fused:
+                c.step_fused(g, n)
+            else:
+                c.accumulate(g, n)
+                c.step()
+        plan = a.get_kernel_plan()
+    case = dict(variant=variant, K=K, M=M, P=P, dtype=str(dtype), order=order, shift=shift, fused=fused, plan=plan)
+    assert plan["pipeline"] == 1 and plan["tiles"] >= 3 * plan["grid"], case
+    assert torch.equal(a.get_params(device="cuda"), d.get_params(device="cuda")), case
+    assert torch.equal(a.get_momentum(device="cuda"), d.get_momentum(device="cuda")), case
+    a.check_guards(); d.check_guards()
+    a.close(); d.close()
+    del flat, g
+    torch.cuda.empty_cache()
