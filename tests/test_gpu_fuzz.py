@@ -100,7 +100,7 @@ def test_random_configuration(case_id):
     ctx.close()
 
 
-@pytest.mark.parametrize("case_id", range(60))
+@pytest.mark.parametrize("case_id", range(100))
 def test_random_differential_between_kernel_families(case_id):
     """The same random problem through the default kernels (bulk-copy pipeline in whichever shape the
     planner picks - box or per-row copies, one to three X buffers, either mixing order - plus the
@@ -159,7 +159,7 @@ def test_random_differential_between_kernel_families(case_id):
     a.close(); d.close()
 
 
-@pytest.mark.parametrize("case_id", range(24))
+@pytest.mark.parametrize("case_id", range(48))
 def test_random_differential_with_many_tiles_per_cta(case_id):
     """The differential test in the persistent regime: about 4100 tiles, so that every CTA of every
     kernel shape (up to nine CTAs per SM) takes three or more tiles - ring phases wrap, X buffers are
