@@ -1091,22 +1091,21 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   const int qpt = t.qpt ? (t.qpt == 2 ? 2 : 1) : (centralized && es == 2 ? 2 : 1);
   // Items of at most 5 KB (M <= 5) leave room for a ninth CTA (4-5 slots each): cfg4 sizes 0.97 -> 1.00, M = 1 / 2 0.55 ->
   // 0.59 / 0.61, M = 5 1.00 -> 1.02, against 1.055 -> 1.045 for 8 KB items, which stay at eight.
-  // Masked accumulate: two CTAs of two groups (cfg3 sizes 1.05, M = 4 0.98-1.00); three when an item is at most 2 KB
-  // of bf16 rows (M = 1, 2: 0.79-0.80 -> 0.92-0.93).
+  // Masked accumulate: two CTAs of two groups (cfg3 sizes 1.05, M = 4 0.98-1.00); three when an item is at most 3 KB
+  // of bf16 rows (M = 1, 2: 0.79-0.80 -> 0.93-0.94; M = 3: 0.92 -> 0.97).
   const int item_bytes = slot_bytes_of(0, T, es, R, row_pad);
   const int ctas = t.ctas_per_sm ? t.ctas_per_sm
                    : centralized ? (es == 2 ? (item_bytes <= 5120 + 128 ? 9 : 8) : 4)
-                                 : (es == 2 && item_bytes <= 2048 + 128 ? 3 : 2);
+                                 : (es == 2 && item_bytes <= 3072 + 128 ? 3 : 2);
   const int budget = kSmemBudget / ctas - 1024;
   int slots = (budget - 512) / slot_bytes_of(0, T, es, R, row_pad);
   if (slots > 16) slots = 16;
   if (!centralized) {
-    // Masked accumulate: about 32 KB of ring per group is the optimum (cfg3 sizes, 8 KB slots, slots per
-    // CTA -> fraction of the measured copy bandwidth: 4 -> 0.86, 6 -> 1.01, 8 -> 1.05, 12 -> 0.91).
-    // (4 KB slots, cfg4 sizes, slots per CTA: 8 -> 0.94, 12 -> 1.00, 14 -> 0.97, 16 -> 0.94: at most 6 per group)
-    int per_group = 32768 / slot_bytes_of(0, T, es, R, row_pad);
-    if (per_group < 2) per_group = 2;
-    if (per_group > 6) per_group = 6;
+    // Masked accumulate: the optimum is a ring of about 100 KB per SM (slots per CTA -> fraction of the measured copy
+    // bandwidth; 8 KB slots, cfg3 sizes: 4 -> 0.86, 6 -> 1.01, 8 -> 1.05, 12 -> 0.91; 6 KB: 8 -> 1.02, 10 -> 0.98; 5 KB: 8 ->
+    // 0.97, 12 -> 0.94; 4 KB, cfg4 sizes: 8 -> 0.94, 12 -> 1.00, 16 -> 0.94; three CTAs, 3 KB: 8 -> 0.97, 12 -> 0.88; 2 KB
+    // and 1 KB: 8 -> 0.90, 12 -> 0.94): four slots per group, six where a slot is at most 4 KB (two CTAs) or 2 KB (three).
+    int per_group = item_bytes <= (ctas == 3 ? 2048 : 4096) + 128 ? 6 : 4;
     if (slots > per_group * groups) slots = per_group * groups;
   }
   if (t.slots && t.slots < slots) slots = t.slots;
