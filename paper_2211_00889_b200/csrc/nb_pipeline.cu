@@ -1100,6 +1100,12 @@ bool plan_stream(const StepArgs &a, int es, bool centralized, PipePlan *plan) {
   const int budget = kSmemBudget / ctas - 1024;
   int slots = (budget - 512) / slot_bytes_of(0, T, es, R, row_pad);
   if (slots > 16) slots = 16;
+  if (centralized && R < a.M) {
+    // learners that need several items per tile do best on a ring of 128 KB per SM (K = 16, bf16, M = 16: three
+    // slots of 8 KB per CTA 1.02, two 1.07; fp32, M = 8: six 1.03, four 1.08); one-item learners use every slot that fits
+    const int cap = 128 * 1024 / (ctas * item_bytes);
+    if (cap >= 2 && slots > cap) slots = cap;
+  }
   if (!centralized) {
     // Masked accumulate: the optimum is a ring of about 100 KB per SM (slots per CTA -> fraction of the measured copy
     // bandwidth; 8 KB slots, cfg3 sizes: 4 -> 0.86, 6 -> 1.01, 8 -> 1.05, 12 -> 0.91; 6 KB: 8 -> 1.02, 10 -> 0.98; 5 KB: 8 ->
