@@ -13,7 +13,9 @@
 //     per tile (the mix needs every neighbour's OLD value while X is updated in place).  The stage
 //     has two buffers, so tile t+1's models load while tile t is consumed; one buffer where two do
 //     not fit (K > 32: the ring keeps the copies going meanwhile); three for the update-then-mix
-//     order (Eq. 4-6), whose averaging pass then runs one tile late;
+//     order (Eq. 4-6), whose averaging pass then runs one tile late.  In that order on one buffer
+//     (template parameter XR) there is no such box at all: x_i travels in learner i's ring item and
+//     the buffer only holds the locally updated models between the two passes of a tile;
 //   * the consumers form NG groups of T/4 threads; group g owns the learners i = g, g+NG, ...
 //     (their updates are independent once the old models are staged) and a PRIVATE ring of slots;
 //     its own producer thread streams that group's "items" into the ring: item = momentum row
